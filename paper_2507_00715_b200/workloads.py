@@ -1,0 +1,161 @@
+"""Seeded synthetic inputs for the EARN attention path.
+
+This module serves both the CUDA path and the CPU oracle and therefore holds
+none of the method's arithmetic: it only draws Q/K/V tensors, prompt lengths
+and beam parents from a seed.  The shapes follow the five workloads the build
+is measured on; the values are i.i.d. N(0,1) with a dual "attention sink"
+bias (Section 1, dual attention sinks; Appendix A.1, Eq. 15) so that the
+first and last prompt positions attract a large share of the attention mass.
+
+Recipe, per layer and per tensor (fresh generator seeded from
+(seed, layer, tensor tag)):
+
+* Q [total, Hq, D], K and V [total, Hkv, D]  ~ N(0,1) in fp32;
+* one unit vector u[kv_head] per workload (from the seed alone);
+* K[first row of every sequence] += 4 u,  K[last row] += 4 u;
+* if ``sink_q_bias``: Q[:, h] += sqrt(D) * u[h // g], which makes the scaled
+  logit of every query toward the two sink keys have mean +4;
+* the result is rounded once to the workload dtype (bf16 or fp32).
+
+Decode-step tensors (one new token per beam) are drawn the same way; beam
+parents are uniform integers in [0, W).
+"""
+from __future__ import annotations
+
+import dataclasses
+import math
+from typing import Dict, Tuple
+
+import numpy as np
+import torch
+
+
+@dataclasses.dataclass(frozen=True)
+class Workload:
+    name: str
+    batch: int
+    n_layers: int          # N
+    split_k: int           # k : layers [0,k) see every token, [k,N) only registers
+    n_q_heads: int         # Hq
+    n_kv_heads: int        # Hkv
+    head_dim: int          # D
+    dtype: str             # "f32" | "bf16"
+    prompt_len: int        # uniform prompt length incl. registers; 0 => ragged
+    len_lo: int = 0        # ragged: lengths uniform in [len_lo, len_hi]
+    len_hi: int = 0
+    r_head: int = 1        # prefix registers
+    r_tail: int = 1        # suffix registers
+    decode_steps: int = 0  # T
+    beams: int = 1         # W
+    seed: int = 0
+    sink_q_bias: bool = True
+
+    @property
+    def group(self) -> int:
+        return self.n_q_heads // self.n_kv_heads
+
+    @property
+    def n_regs(self) -> int:
+        return self.r_head + self.r_tail
+
+    @property
+    def torch_dtype(self) -> torch.dtype:
+        return torch.float32 if self.dtype == "f32" else torch.bfloat16
+
+    def replace(self, **kw) -> "Workload":
+        return dataclasses.replace(self, **kw)
+
+
+CONFIGS: Dict[str, Workload] = {
+    "tiny": Workload("tiny", batch=1, n_layers=4, split_k=2, n_q_heads=4, n_kv_heads=4, head_dim=64,
+                     dtype="f32", prompt_len=256, r_head=4, r_tail=4, decode_steps=8, beams=1, seed=1),
+    "1p5b": Workload("1p5b", batch=32, n_layers=28, split_k=4, n_q_heads=12, n_kv_heads=2, head_dim=128,
+                     dtype="bf16", prompt_len=512, r_head=8, r_tail=8, decode_steps=16, beams=1, seed=2),
+    "7b": Workload("7b", batch=64, n_layers=32, split_k=8, n_q_heads=32, n_kv_heads=8, head_dim=128,
+                   dtype="bf16", prompt_len=1024, r_head=16, r_tail=16, decode_steps=20, beams=1, seed=3),
+    "long": Workload("long", batch=8, n_layers=32, split_k=8, n_q_heads=32, n_kv_heads=8, head_dim=128,
+                     dtype="bf16", prompt_len=4096, r_head=16, r_tail=16, decode_steps=20, beams=1, seed=4),
+    "ragged": Workload("ragged", batch=128, n_layers=32, split_k=8, n_q_heads=32, n_kv_heads=8, head_dim=128,
+                       dtype="bf16", prompt_len=0, len_lo=128, len_hi=2048, r_head=16, r_tail=16,
+                       decode_steps=20, beams=10, seed=5),
+}
+LONG_SPLIT_SWEEP = (2, 4, 8, 16)
+
+_TAG = {"q": 1, "k": 2, "v": 3, "dq": 4, "dk": 5, "dv": 6, "len": 7, "u": 8, "parent": 9}
+
+
+def _seed_for(w: Workload, tag: str, layer: int = 0, step: int = 0) -> int:
+    # a plain mixed-radix key; distinct (seed, tag, layer, step) give distinct streams
+    return ((w.seed * 16 + _TAG[tag]) * 4096 + layer) * 4096 + step
+
+
+def seqlens(w: Workload) -> np.ndarray:
+    """Prompt length of every sequence, registers included (int32 [batch])."""
+    if w.prompt_len > 0:
+        return np.full((w.batch,), w.prompt_len, dtype=np.int32)
+    rng = np.random.Generator(np.random.Philox(_seed_for(w, "len")))
+    return rng.integers(w.len_lo, w.len_hi + 1, size=w.batch).astype(np.int32)
+
+
+def cu_seqlens(w: Workload) -> np.ndarray:
+    """Exclusive prefix sum of :func:`seqlens` (int32 [batch+1])."""
+    out = np.zeros(w.batch + 1, dtype=np.int32)
+    np.cumsum(seqlens(w), out=out[1:])
+    return out
+
+
+def sink_direction(w: Workload) -> torch.Tensor:
+    """One fp32 unit vector per kv head, [Hkv, D], CPU."""
+    g = torch.Generator()
+    g.manual_seed(_seed_for(w, "u"))
+    u = torch.randn(w.n_kv_heads, w.head_dim, generator=g, dtype=torch.float32)
+    return u / u.norm(dim=1, keepdim=True)
+
+
+def _randn(shape, seed: int, device) -> torch.Tensor:
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    return torch.randn(shape, generator=g, device=device, dtype=torch.float32)
+
+
+def layer_qkv(w: Workload, layer: int, device="cpu") -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    """Packed prompt tensors of one layer: Q [total,Hq,D], K,V [total,Hkv,D] in the workload dtype."""
+    cu = cu_seqlens(w)
+    total = int(cu[-1])
+    u = sink_direction(w).to(device)
+    q = _randn((total, w.n_q_heads, w.head_dim), _seed_for(w, "q", layer), device)
+    k = _randn((total, w.n_kv_heads, w.head_dim), _seed_for(w, "k", layer), device)
+    v = _randn((total, w.n_kv_heads, w.head_dim), _seed_for(w, "v", layer), device)
+    first = torch.as_tensor(cu[:-1].astype(np.int64), device=device)
+    last = torch.as_tensor((cu[1:] - 1).astype(np.int64), device=device)
+    k[first] += 4.0 * u
+    # a one-token sequence gets the bias once per role, as the recipe states it
+    k[last] += 4.0 * u
+    if w.sink_q_bias:
+        q += math.sqrt(w.head_dim) * u.repeat_interleave(w.group, dim=0)
+    dt = w.torch_dtype
+    return q.to(dt), k.to(dt), v.to(dt)
+
+
+def decode_qkv(w: Workload, layer: int, step: int, device="cpu"):
+    """One decode step (1-based): q [B*W,Hq,D], k_new and v_new [B*W,Hkv,D]."""
+    rows = w.batch * w.beams
+    u = sink_direction(w).to(device)
+    q = _randn((rows, w.n_q_heads, w.head_dim), _seed_for(w, "dq", layer, step), device)
+    k = _randn((rows, w.n_kv_heads, w.head_dim), _seed_for(w, "dk", layer, step), device)
+    v = _randn((rows, w.n_kv_heads, w.head_dim), _seed_for(w, "dv", layer, step), device)
+    if w.sink_q_bias:
+        q += math.sqrt(w.head_dim) * u.repeat_interleave(w.group, dim=0)
+    dt = w.torch_dtype
+    return q.to(dt), k.to(dt), v.to(dt)
+
+
+def beam_parents(w: Workload, step: int) -> np.ndarray:
+    """Parent beam (index within the sequence, in [0,W)) of every beam at a decode step (1-based).
+
+    Step 1 has no history to inherit; its parents are the identity.  int32 [B*W].
+    """
+    if step <= 1 or w.beams == 1:
+        return np.tile(np.arange(w.beams, dtype=np.int32), w.batch)
+    rng = np.random.Generator(np.random.Philox(_seed_for(w, "parent", 0, step)))
+    return rng.integers(0, w.beams, size=w.batch * w.beams).astype(np.int32)
