@@ -1,0 +1,160 @@
+/*
+ * earn.h — C ABI of the EARN attention hot path for NVIDIA B200 (sm_100a).
+ *
+ * EARN runs the first k decoder layers over every prompt token and the
+ * remaining N-k layers over the register tokens (a few learnable tokens at the
+ * head and tail of the prompt) plus the generated tokens only (Section 3.2,
+ * "Inference").  This library is the attention part of that pipeline:
+ *
+ *   layers l <  k : earn_prefill_attn                       (prefill)   earn_decode_attn with k_full/v_full (decode)
+ *   layers l >= k : earn_compact_kv -> earn_register_attn    (prefill)   earn_decode_attn over the compact cache (decode)
+ *
+ * Layers are 0-indexed: 0..k-1 are full layers, k..N-1 register layers.
+ *
+ * Conventions for every call
+ *   - "device" pointers are CUDA device memory owned by the caller; "host" pointers are
+ *     ordinary host memory.  Nothing is retained after a call returns except where stated.
+ *   - tensors are dense, innermost dimension contiguous, base addresses 16-byte aligned.
+ *   - dtype EARN_BF16: elements are bfloat16, arithmetic is fp32 (softmax, accumulation),
+ *     outputs are rounded once to bfloat16.  EARN_F32: fp32 in and out (debug path).
+ *   - `stream` is a cudaStream_t passed as an opaque pointer (NULL = legacy default stream).
+ *     Calls only enqueue work on it; they do not synchronise and allocate no device memory
+ *     (workspace comes from the caller), except earn_device_status which synchronises.
+ *   - every argument check happens on the host before anything is launched; a call that
+ *     returns a status other than EARN_OK has launched nothing, except EARN_ERR_CUDA, which
+ *     reports a failed launch.  Nothing throws or exits.
+ */
+#ifndef EARN_H_
+#define EARN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void* earn_stream_t;
+
+typedef enum {
+  EARN_OK = 0,
+  EARN_ERR_INVALID_ARG = 1, /* null/misaligned pointer, bad shape, layer on the wrong side of k, R > L_b ... */
+  EARN_ERR_UNSUPPORTED = 2, /* legal request this build has no kernel for (e.g. head_dim not in {64,128}) */
+  EARN_ERR_WORKSPACE = 3,   /* workspace NULL or smaller than earn_workspace_bytes() */
+  EARN_ERR_CUDA = 4,        /* the CUDA runtime reported an error at launch */
+  EARN_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (read back by earn_device_status) */
+} earn_status_t;
+
+typedef enum { EARN_F32 = 0, EARN_BF16 = 1 } earn_dtype_t;
+
+#define EARN_PAGE_TOKENS 16 /* tokens per page of the compact register cache */
+
+/* Model shape.  Section 3.3 notation: N layers, split k, n_h heads, d_a per-head dimension. */
+typedef struct {
+  int32_t n_layers;    /* N  > 0 */
+  int32_t split_k;     /* k, 0 <= k <= N; k = N is a vanilla model, k = 0 compacts at the first layer */
+  int32_t n_q_heads;   /* Hq, multiple of n_kv_heads */
+  int32_t n_kv_heads;  /* Hkv */
+  int32_t head_dim;    /* D in {64, 128} */
+  int32_t dtype;       /* earn_dtype_t */
+  float softmax_scale; /* 0 => 1/sqrt(head_dim), the scale of Eq. 3 */
+} earn_model_t;
+
+/* One batch of prompts, packed back to back (no padding tokens exist).  Eq. 5: every sequence is
+ * [prefix registers; prompt; suffix registers]; its length L_b counts the registers. */
+typedef struct {
+  int32_t batch;                  /* B >= 0 */
+  int32_t total_tokens;           /* sum of L_b */
+  int32_t max_seqlen;             /* max L_b */
+  const int32_t* cu_seqlens;      /* device [B+1], exclusive prefix sum of L_b */
+  const int32_t* cu_seqlens_host; /* host   [B+1], the same values (used for validation and scheduling) */
+  int32_t n_head_reg;             /* r_h >= 0 prefix registers = the first r_h positions of every sequence */
+  int32_t n_tail_reg;             /* r_t >= 0 suffix registers = the last r_t positions; r_h + r_t <= every L_b */
+} earn_batch_t;
+
+/* KV cache of ONE register layer (l >= k) plus the generated-token cache of any layer.
+ * Shared segment: the R = r_h + r_t register rows of every sequence in pages of EARN_PAGE_TOKENS
+ * tokens, written once by earn_compact_kv and read by all beams of the sequence.
+ * Private segment: the tokens generated so far, one slab per beam. */
+typedef struct {
+  void* k_shared;             /* device [n_pages, 16, Hkv, D]; may be NULL for a layer < k */
+  void* v_shared;             /* device, same shape */
+  const int32_t* block_table; /* device [B, pages_per_seq] page numbers, or NULL: page p of sequence b is b*pages_per_seq+p */
+  int32_t pages_per_seq;      /* >= ceil(R / 16) */
+  int32_t n_pages;            /* pages allocated in k_shared / v_shared (bounds the block table) */
+  void* k_priv;               /* device [B*beams, max_new, Hkv, D] generated keys; row (j, t) is written at step t+1 by beam j */
+  void* v_priv;               /* device, same shape */
+  const int32_t* lineage;     /* device [B*beams, max_new] or NULL (identity): lineage[j][t] = slab holding token t of the
+                                 history of beam j, maintained by earn_beam_reparent */
+  int32_t beams;              /* W >= 1 */
+  int32_t max_new;            /* T: capacity of the private segment in tokens */
+  int32_t* reg_idx;           /* device [B, R] or NULL: earn_compact_kv writes the gathered source positions here */
+} earn_cache_t;
+
+/* Bytes of caller-provided scratch that cover every call below for this model, batch and beam
+ * width (0 is never returned; the first 256 bytes hold the device status word).  Host only. */
+size_t earn_workspace_bytes(const earn_model_t* model, const earn_batch_t* batch, int32_t beams);
+
+/* Clears the device status word.  Call once after allocating the workspace (asynchronous). */
+earn_status_t earn_workspace_init(void* workspace, size_t workspace_bytes, earn_stream_t stream);
+
+/* Synchronises `stream` and returns the device status word of the workspace: EARN_OK, or
+ * EARN_ERR_TIMEOUT if a bounded wait inside a kernel ran out since earn_workspace_init. */
+earn_status_t earn_device_status(const void* workspace, earn_stream_t stream);
+
+/* Step 1 — full causal attention of a layer l < k over every prompt token
+ * (Section 3.2 "Full Computation Process"; Eq. 3 with the causal mask of a decoder-only model):
+ *   O[i,h] = sum_{j<=i} softmax_j( Q[i,h].K[j,h/g] * scale ) V[j,h/g]   within each sequence, g = Hq/Hkv.
+ * q,o: device [total_tokens, Hq, D]; k,v: device [total_tokens, Hkv, D] (read in place later by decode).
+ * lse_or_null: device fp32 [Hq, total_tokens], natural-log softmax denominators, or NULL.
+ * Errors: layer outside [0,k) -> INVALID_ARG. */
+earn_status_t earn_prefill_attn(const earn_model_t* model, const earn_batch_t* batch, int32_t layer,
+                                const void* q, const void* k, const void* v, void* o, float* lse_or_null,
+                                void* workspace, size_t workspace_bytes, earn_stream_t stream);
+
+/* Step 2 — keep only the register rows at a layer l >= k
+ * (Section 3.2 "Register-Focused Process": X = [prefix; Prompt; suffix] -> X' = [prefix; suffix]).
+ * For sequence b the source positions are idx_b = (0..r_h-1, L_b-r_t..L_b-1); row m of the compact cache
+ * is a bit copy of row idx_b[m] of k and v.  If q_or_null is given, the same rows of q go to
+ * q_reg_or_null (device [B, R, Hq, D]), ready for earn_register_attn.  cache->reg_idx (if not NULL)
+ * receives idx.  Errors: layer outside [k,N), R > some L_b, page table too small -> INVALID_ARG. */
+earn_status_t earn_compact_kv(const earn_model_t* model, const earn_batch_t* batch, int32_t layer,
+                              const void* k, const void* v, const void* q_or_null, void* q_reg_or_null,
+                              const earn_cache_t* cache, earn_stream_t stream);
+
+/* Step 3 — attention of a layer l >= k during prefill: causal attention among the R register tokens of
+ * each sequence in the order [prefix; suffix] (Section 3.2, training rule "only register ... tokens
+ * participate", and the inference rule above).  q_reg, o_reg: device [B, R, Hq, D]. */
+earn_status_t earn_register_attn(const earn_model_t* model, const earn_batch_t* batch, int32_t layer,
+                                 const void* q_reg, const earn_cache_t* cache, void* o_reg,
+                                 void* workspace, size_t workspace_bytes, earn_stream_t stream);
+
+/* Step 4 — one decode step of one layer (Eq. 4: append K_t, V_t, then attend over K_{1:t}, self included).
+ * step is 1-based; beam j = b*W + w.  k_new/v_new (device [B*W, Hkv, D]) are stored at row (j, step-1) of the
+ * private segment; q, o: device [B*W, Hq, D].  Keys seen by beam j:
+ *   layer >= k : the R compact register rows of sequence b, then the step generated tokens of its lineage;
+ *   layer <  k : all L_b prompt rows of sequence b read in place from k_full/v_full (device, packed like
+ *                earn_prefill_attn's k and v; required), then the generated tokens.
+ * Errors: step outside [1, max_new], missing k_full for a layer < k -> INVALID_ARG. */
+earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, int32_t step,
+                               const void* q, const void* k_new, const void* v_new,
+                               const void* k_full_or_null, const void* v_full_or_null,
+                               const earn_cache_t* cache, void* o,
+                               void* workspace, size_t workspace_bytes, earn_stream_t stream);
+
+/* Beam search bookkeeping between decode steps (Appendix A.3 uses beam search; the cache sharing is this
+ * library's design): before step `step` (>= 2), beam j continues the history of beam parent[j] (an index in
+ * [0,W) within its own sequence).  No K/V moves: lineage_out[j][t] = lineage_in[b*W+parent[j]][t] for
+ * t < step-1 and lineage_out[j][step-1] = j.  lineage_in NULL means the identity table.  One table serves
+ * all layers of a step.  lineage_in and lineage_out must not alias.  All pointers device. */
+earn_status_t earn_beam_reparent(int32_t batch, int32_t beams, int32_t max_new, int32_t step,
+                                 const int32_t* parent, const int32_t* lineage_in_or_null,
+                                 int32_t* lineage_out, earn_stream_t stream);
+
+const char* earn_status_string(earn_status_t status);
+int32_t earn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EARN_H_ */

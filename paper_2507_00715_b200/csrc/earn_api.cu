@@ -1,0 +1,264 @@
+// C-ABI entry points: host-side validation, workspace layout and kernel dispatch.
+#include <cstdio>
+#include <cstring>
+
+#include "earn_common.cuh"
+
+namespace earn {
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static earn_status_t check_model(const earn_model_t* m) {
+  if (m == nullptr) return EARN_ERR_INVALID_ARG;
+  if (m->n_layers <= 0 || m->split_k < 0 || m->split_k > m->n_layers) return EARN_ERR_INVALID_ARG;
+  if (m->n_q_heads <= 0 || m->n_kv_heads <= 0 || m->n_q_heads % m->n_kv_heads != 0) return EARN_ERR_INVALID_ARG;
+  if (m->dtype != EARN_F32 && m->dtype != EARN_BF16) return EARN_ERR_INVALID_ARG;
+  if (!(m->softmax_scale >= 0.f)) return EARN_ERR_INVALID_ARG;
+  if (m->head_dim <= 0) return EARN_ERR_INVALID_ARG;
+  if (m->head_dim != 64 && m->head_dim != 128) return EARN_ERR_UNSUPPORTED;
+  if (m->n_q_heads > 65535) return EARN_ERR_UNSUPPORTED;
+  return EARN_OK;
+}
+
+static earn_status_t check_batch(const earn_batch_t* b) {
+  if (b == nullptr) return EARN_ERR_INVALID_ARG;
+  if (b->batch < 0 || b->total_tokens < 0 || b->max_seqlen < 0) return EARN_ERR_INVALID_ARG;
+  if (b->n_head_reg < 0 || b->n_tail_reg < 0) return EARN_ERR_INVALID_ARG;
+  if (b->batch > 65535) return EARN_ERR_UNSUPPORTED;
+  if (b->batch == 0) return b->total_tokens == 0 ? EARN_OK : EARN_ERR_INVALID_ARG;
+  if (b->cu_seqlens == nullptr || b->cu_seqlens_host == nullptr) return EARN_ERR_INVALID_ARG;
+  const int32_t* cu = b->cu_seqlens_host;
+  if (cu[0] != 0 || cu[b->batch] != b->total_tokens) return EARN_ERR_INVALID_ARG;
+  int mx = 0;
+  for (int i = 0; i < b->batch; ++i) {
+    int len = cu[i + 1] - cu[i];
+    if (len < 0) return EARN_ERR_INVALID_ARG;
+    if (len < b->n_head_reg + b->n_tail_reg) return EARN_ERR_INVALID_ARG;   // registers are rows of the sequence
+    mx = len > mx ? len : mx;
+  }
+  if (mx > b->max_seqlen) return EARN_ERR_INVALID_ARG;
+  return EARN_OK;
+}
+
+static float scale_of(const earn_model_t* m) {
+  return m->softmax_scale > 0.f ? m->softmax_scale : 1.0f / sqrtf((float)m->head_dim);
+}
+static size_t elem_size(const earn_model_t* m) { return m->dtype == EARN_F32 ? 4 : 2; }
+
+DecodePlan make_decode_plan(const earn_model_t& m, const earn_batch_t& b, int beams, int max_shared_len) {
+  DecodePlan p{};
+  p.rows = beams * (m.n_q_heads / m.n_kv_heads);
+  p.row_tiles = (p.rows + kDecodeRows - 1) / kDecodeRows;
+  p.rows_pad = p.row_tiles * kDecodeRows;
+  if (max_shared_len <= 0 || b.batch == 0) { p.chunk = 64; p.n_splits = 0; return p; }
+  // enough CTAs to cover the SMs a few times over, but no more splits than that needs
+  const long units = (long)b.batch * m.n_kv_heads * p.row_tiles;
+  const long want = 4L * 148;
+  long splits = (want + units - 1) / units;
+  long max_splits = (max_shared_len + 63) / 64;
+  if (splits > max_splits) splits = max_splits;
+  if (splits < 1) splits = 1;
+  p.chunk = (int)round_up((size_t)((max_shared_len + splits - 1) / splits), 64);
+  p.n_splits = (max_shared_len + p.chunk - 1) / p.chunk;
+  return p;
+}
+
+size_t decode_partial_floats(const earn_model_t& m, const earn_batch_t& b, const DecodePlan& p) {
+  return (size_t)b.batch * m.n_kv_heads * p.n_splits * p.rows_pad * (size_t)(m.head_dim + 1);
+}
+
+static size_t workspace_need(const earn_model_t* m, const earn_batch_t* b, int beams) {
+  DecodePlan full = make_decode_plan(*m, *b, beams, b->max_seqlen);
+  DecodePlan reg = make_decode_plan(*m, *b, beams, b->n_head_reg + b->n_tail_reg);
+  size_t f = decode_partial_floats(*m, *b, full), r = decode_partial_floats(*m, *b, reg);
+  return kStatusBytes + round_up(sizeof(float) * (f > r ? f : r), 256) + 256;
+}
+
+static earn_status_t check_cache_shared(const earn_model_t* m, const earn_batch_t* b, const earn_cache_t* c) {
+  const int R = b->n_head_reg + b->n_tail_reg;
+  if (c == nullptr) return EARN_ERR_INVALID_ARG;
+  if (R == 0) return EARN_OK;
+  if (c->k_shared == nullptr || c->v_shared == nullptr || !aligned16(c->k_shared) || !aligned16(c->v_shared))
+    return EARN_ERR_INVALID_ARG;
+  const int need = (R + EARN_PAGE_TOKENS - 1) / EARN_PAGE_TOKENS;
+  if (c->pages_per_seq < need) return EARN_ERR_INVALID_ARG;
+  if (c->block_table == nullptr && (int64_t)c->n_pages < (int64_t)b->batch * c->pages_per_seq) return EARN_ERR_INVALID_ARG;
+  if (c->n_pages <= 0) return EARN_ERR_INVALID_ARG;
+  (void)m;
+  return EARN_OK;
+}
+
+static KeySource paged_source(const earn_batch_t* b, const earn_cache_t* c) {
+  KeySource s{};
+  s.k = c->k_shared; s.v = c->v_shared;
+  s.block_table = c->block_table; s.pages_per_seq = c->pages_per_seq; s.n_pages = c->n_pages;
+  s.paged = 1; s.n_regs = b->n_head_reg + b->n_tail_reg;
+  return s;
+}
+
+}  // namespace earn
+
+using namespace earn;
+
+extern "C" {
+
+int32_t earn_version(void) { return 100; }
+
+const char* earn_status_string(earn_status_t s) {
+  switch (s) {
+    case EARN_OK: return "ok";
+    case EARN_ERR_INVALID_ARG: return "invalid argument";
+    case EARN_ERR_UNSUPPORTED: return "unsupported configuration";
+    case EARN_ERR_WORKSPACE: return "workspace missing or too small";
+    case EARN_ERR_CUDA: return "CUDA error at launch";
+    case EARN_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+size_t earn_workspace_bytes(const earn_model_t* model, const earn_batch_t* batch, int32_t beams) {
+  if (check_model(model) != EARN_OK || batch == nullptr || beams < 1) return kStatusBytes;
+  return workspace_need(model, batch, beams);
+}
+
+earn_status_t earn_workspace_init(void* workspace, size_t workspace_bytes, earn_stream_t stream) {
+  if (workspace == nullptr || workspace_bytes < (size_t)kStatusBytes || !aligned16(workspace)) return EARN_ERR_WORKSPACE;
+  return cudaMemsetAsync(workspace, 0, kStatusBytes, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+}
+
+earn_status_t earn_device_status(const void* workspace, earn_stream_t stream) {
+  if (workspace == nullptr) return EARN_ERR_WORKSPACE;
+  int32_t word = 0;
+  if (cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
+    return EARN_ERR_CUDA;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return EARN_ERR_CUDA;
+  return word == 0 ? EARN_OK : EARN_ERR_TIMEOUT;
+}
+
+earn_status_t earn_prefill_attn(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, const void* q,
+                                const void* k, const void* v, void* o, float* lse_or_null, void* workspace,
+                                size_t workspace_bytes, earn_stream_t stream) {
+  earn_status_t s = check_model(model);
+  if (s != EARN_OK) return s;
+  s = check_batch(batch);
+  if (s != EARN_OK) return s;
+  if (layer < 0 || layer >= model->split_k) return EARN_ERR_INVALID_ARG;
+  if (batch->total_tokens == 0) return EARN_OK;
+  if (!q || !k || !v || !o || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return EARN_ERR_INVALID_ARG;
+  if (lse_or_null && !aligned16(lse_or_null)) return EARN_ERR_INVALID_ARG;
+  if (workspace == nullptr || workspace_bytes < (size_t)kStatusBytes) return EARN_ERR_WORKSPACE;
+  PrefillArgs a{};
+  a.q = q; a.k = k; a.v = v; a.o = o; a.lse = lse_or_null;
+  a.cu_seqlens = batch->cu_seqlens;
+  a.batch = batch->batch; a.max_seqlen = batch->max_seqlen;
+  a.Hq = model->n_q_heads; a.Hkv = model->n_kv_heads; a.D = model->head_dim; a.dtype = model->dtype;
+  a.scale = scale_of(model);
+  return launch_prefill_simt(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+}
+
+earn_status_t earn_compact_kv(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, const void* k,
+                              const void* v, const void* q_or_null, void* q_reg_or_null, const earn_cache_t* cache,
+                              earn_stream_t stream) {
+  earn_status_t s = check_model(model);
+  if (s != EARN_OK) return s;
+  s = check_batch(batch);
+  if (s != EARN_OK) return s;
+  if (layer < model->split_k || layer >= model->n_layers) return EARN_ERR_INVALID_ARG;
+  s = check_cache_shared(model, batch, cache);
+  if (s != EARN_OK) return s;
+  const int R = batch->n_head_reg + batch->n_tail_reg;
+  if (R == 0 || batch->batch == 0) return EARN_OK;
+  if (!k || !v || !aligned16(k) || !aligned16(v)) return EARN_ERR_INVALID_ARG;
+  if ((q_or_null == nullptr) != (q_reg_or_null == nullptr)) return EARN_ERR_INVALID_ARG;
+  if (q_or_null && (!aligned16(q_or_null) || !aligned16(q_reg_or_null))) return EARN_ERR_INVALID_ARG;
+  CompactArgs a{};
+  a.k = k; a.v = v; a.q = q_or_null;
+  a.k_shared = cache->k_shared; a.v_shared = cache->v_shared; a.q_reg = q_reg_or_null;
+  a.cu_seqlens = batch->cu_seqlens; a.block_table = cache->block_table; a.reg_idx = cache->reg_idx;
+  a.pages_per_seq = cache->pages_per_seq; a.n_pages = cache->n_pages; a.batch = batch->batch;
+  a.r_head = batch->n_head_reg; a.r_tail = batch->n_tail_reg;
+  a.kv_row_bytes = (int)(model->n_kv_heads * model->head_dim * elem_size(model));
+  a.q_row_bytes = (int)(model->n_q_heads * model->head_dim * elem_size(model));
+  return launch_compact(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+}
+
+earn_status_t earn_register_attn(const earn_model_t* model, const earn_batch_t* batch, int32_t layer,
+                                 const void* q_reg, const earn_cache_t* cache, void* o_reg, void* workspace,
+                                 size_t workspace_bytes, earn_stream_t stream) {
+  earn_status_t s = check_model(model);
+  if (s != EARN_OK) return s;
+  s = check_batch(batch);
+  if (s != EARN_OK) return s;
+  if (layer < model->split_k || layer >= model->n_layers) return EARN_ERR_INVALID_ARG;
+  s = check_cache_shared(model, batch, cache);
+  if (s != EARN_OK) return s;
+  const int R = batch->n_head_reg + batch->n_tail_reg;
+  if (R == 0 || batch->batch == 0) return EARN_OK;
+  if (!q_reg || !o_reg || !aligned16(q_reg) || !aligned16(o_reg)) return EARN_ERR_INVALID_ARG;
+  if (workspace == nullptr || workspace_bytes < (size_t)kStatusBytes) return EARN_ERR_WORKSPACE;
+  RegisterArgs a{};
+  a.q_reg = q_reg; a.o_reg = o_reg;
+  a.src = paged_source(batch, cache);
+  a.batch = batch->batch; a.R = R;
+  a.Hq = model->n_q_heads; a.Hkv = model->n_kv_heads; a.D = model->head_dim; a.dtype = model->dtype;
+  a.scale = scale_of(model);
+  return launch_register_simt(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+}
+
+earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, int32_t step,
+                               const void* q, const void* k_new, const void* v_new, const void* k_full_or_null,
+                               const void* v_full_or_null, const earn_cache_t* cache, void* o, void* workspace,
+                               size_t workspace_bytes, earn_stream_t stream) {
+  earn_status_t s = check_model(model);
+  if (s != EARN_OK) return s;
+  s = check_batch(batch);
+  if (s != EARN_OK) return s;
+  if (layer < 0 || layer >= model->n_layers || cache == nullptr) return EARN_ERR_INVALID_ARG;
+  if (cache->beams < 1 || cache->max_new < 1 || step < 1 || step > cache->max_new) return EARN_ERR_INVALID_ARG;
+  if ((int64_t)batch->batch * cache->beams > 65535) return EARN_ERR_UNSUPPORTED;
+  if (batch->batch == 0) return EARN_OK;
+  const bool early = layer < model->split_k;
+  if (early) {
+    if (!k_full_or_null || !v_full_or_null || !aligned16(k_full_or_null) || !aligned16(v_full_or_null))
+      return EARN_ERR_INVALID_ARG;
+  } else {
+    s = check_cache_shared(model, batch, cache);
+    if (s != EARN_OK) return s;
+  }
+  if (!q || !k_new || !v_new || !o || !cache->k_priv || !cache->v_priv) return EARN_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(o) || !aligned16(cache->k_priv) ||
+      !aligned16(cache->v_priv))
+    return EARN_ERR_INVALID_ARG;
+  if (workspace == nullptr || !aligned16(workspace) || workspace_bytes < workspace_need(model, batch, cache->beams))
+    return EARN_ERR_WORKSPACE;
+
+  DecodeArgs a{};
+  a.q = q; a.k_new = k_new; a.v_new = v_new; a.o = o;
+  if (early) {
+    a.src.k = k_full_or_null; a.src.v = v_full_or_null; a.src.cu_seqlens = batch->cu_seqlens; a.src.paged = 0;
+  } else {
+    a.src = paged_source(batch, cache);
+  }
+  a.cu_seqlens = batch->cu_seqlens;
+  a.k_priv = cache->k_priv; a.v_priv = cache->v_priv; a.lineage = cache->lineage;
+  a.plan = make_decode_plan(*model, *batch, cache->beams,
+                            early ? batch->max_seqlen : batch->n_head_reg + batch->n_tail_reg);
+  a.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) + kStatusBytes);
+  a.part_lse = a.part_o + (size_t)batch->batch * model->n_kv_heads * a.plan.n_splits * a.plan.rows_pad * model->head_dim;
+  a.batch = batch->batch; a.beams = cache->beams; a.max_new = cache->max_new; a.step = step;
+  a.Hq = model->n_q_heads; a.Hkv = model->n_kv_heads; a.D = model->head_dim; a.dtype = model->dtype;
+  a.scale = scale_of(model);
+  return launch_decode_simt(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+}
+
+earn_status_t earn_beam_reparent(int32_t batch, int32_t beams, int32_t max_new, int32_t step, const int32_t* parent,
+                                 const int32_t* lineage_in_or_null, int32_t* lineage_out, earn_stream_t stream) {
+  if (batch < 0 || beams < 1 || max_new < 1 || step < 1 || step > max_new) return EARN_ERR_INVALID_ARG;
+  if (batch == 0) return EARN_OK;
+  if (parent == nullptr || lineage_out == nullptr || lineage_out == lineage_in_or_null) return EARN_ERR_INVALID_ARG;
+  return launch_beam_reparent(batch, beams, max_new, step, parent, lineage_in_or_null, lineage_out,
+                              (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,125 @@
+// Shared declarations of the CUDA side of the EARN attention library (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "earn.h"
+
+namespace earn {
+
+constexpr int kStatusBytes = 256;   // head of the workspace: device status word (+ padding)
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// Where the keys/values a query may see before the generated tokens live ("shared segment").
+struct KeySource {
+  const void* k;
+  const void* v;
+  const int32_t* cu_seqlens;   // packed source: row (b, j) is row cu_seqlens[b] + j of [total, Hkv, D]
+  const int32_t* block_table;  // paged source: [B, pages_per_seq] or null (identity)
+  int pages_per_seq;
+  int n_pages;                 // paged: pages allocated (page numbers are clamped to it)
+  int paged;                   // 0: packed prompt K/V, 1: compact register cache in pages of 16 tokens
+  int n_regs;                  // paged: rows per sequence (R)
+};
+
+__device__ __forceinline__ int64_t key_row(const KeySource& s, int b, int j) {
+  if (s.paged) {
+    int page = j / EARN_PAGE_TOKENS;
+    int phys = s.block_table ? s.block_table[b * s.pages_per_seq + page] : b * s.pages_per_seq + page;
+    phys = min(max(phys, 0), s.n_pages - 1);   // a corrupt table reads a wrong page, never outside the cache
+    return (int64_t)phys * EARN_PAGE_TOKENS + (j % EARN_PAGE_TOKENS);
+  }
+  return (int64_t)s.cu_seqlens[b] + j;
+}
+
+// How split-KV decode divides the shared segment; the same numbers size the workspace.
+struct DecodePlan {
+  int rows;        // W * g query rows per (sequence, kv head)
+  int row_tiles;   // tiles of kDecodeRows rows
+  int rows_pad;    // row_tiles * kDecodeRows
+  int chunk;       // keys per split (multiple of 64)
+  int n_splits;    // ceil(max shared length / chunk); 0 when the shared segment is empty
+};
+constexpr int kDecodeRows = 16;
+DecodePlan make_decode_plan(const earn_model_t& m, const earn_batch_t& b, int beams, int max_shared_len);
+size_t decode_partial_floats(const earn_model_t& m, const earn_batch_t& b, const DecodePlan& p);
+
+// ---- launchers (one per .cu file); all return cudaGetLastError() of their launches ----
+struct PrefillArgs {
+  const void *q, *k, *v;
+  void* o;
+  float* lse;
+  const int32_t* cu_seqlens;
+  int batch, max_seqlen, Hq, Hkv, D, dtype;
+  float scale;
+};
+cudaError_t launch_prefill_simt(const PrefillArgs& a, cudaStream_t st);
+
+struct RegisterArgs {
+  const void* q_reg;
+  void* o_reg;
+  KeySource src;
+  int batch, R, Hq, Hkv, D, dtype;
+  float scale;
+};
+cudaError_t launch_register_simt(const RegisterArgs& a, cudaStream_t st);
+
+struct DecodeArgs {
+  const void *q, *k_new, *v_new;
+  void* o;
+  KeySource src;
+  const int32_t* cu_seqlens;   // device, for the shared length of a packed source
+  void *k_priv, *v_priv;
+  const int32_t* lineage;
+  float* part_o;               // [B, Hkv, n_splits, rows_pad, D]
+  float* part_lse;             // [B, Hkv, n_splits, rows_pad]  (log2 domain)
+  DecodePlan plan;
+  int batch, beams, max_new, step, Hq, Hkv, D, dtype;
+  float scale;
+};
+cudaError_t launch_decode_simt(const DecodeArgs& a, cudaStream_t st);
+
+struct CompactArgs {
+  const void *k, *v, *q;
+  void *k_shared, *v_shared, *q_reg;
+  const int32_t* cu_seqlens;
+  const int32_t* block_table;
+  int32_t* reg_idx;
+  int pages_per_seq, n_pages, batch, r_head, r_tail, kv_row_bytes, q_row_bytes;
+};
+cudaError_t launch_compact(const CompactArgs& a, cudaStream_t st);
+
+cudaError_t launch_beam_reparent(int batch, int beams, int max_new, int step, const int32_t* parent,
+                                 const int32_t* lineage_in, int32_t* lineage_out, cudaStream_t st);
+
+// ---- element helpers ----
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+  static __device__ __forceinline__ void load4(const float* p, float (&x)[4]) {
+    float4 t = *reinterpret_cast<const float4*>(p);
+    x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
+  }
+  static __device__ __forceinline__ void store4(float* p, const float (&x)[4]) {
+    *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
+  }
+};
+template <> struct Elem<__nv_bfloat16> {
+  static __device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&x)[4]) {
+    uint2 t = *reinterpret_cast<const uint2*>(p);
+    __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162*>(&t.x);
+    __nv_bfloat162 b = *reinterpret_cast<__nv_bfloat162*>(&t.y);
+    x[0] = __low2float(a); x[1] = __high2float(a); x[2] = __low2float(b); x[3] = __high2float(b);
+  }
+  static __device__ __forceinline__ void store4(__nv_bfloat16* p, const float (&x)[4]) {
+    __nv_bfloat162 a = __floats2bfloat162_rn(x[0], x[1]);
+    __nv_bfloat162 b = __floats2bfloat162_rn(x[2], x[3]);
+    uint2 t;
+    t.x = *reinterpret_cast<uint32_t*>(&a);
+    t.y = *reinterpret_cast<uint32_t*>(&b);
+    *reinterpret_cast<uint2*>(p) = t;
+  }
+};
+
+}  // namespace earn

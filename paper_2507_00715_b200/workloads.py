@@ -49,6 +49,7 @@ class Workload:
     beams: int = 1         # W
     seed: int = 0
     sink_q_bias: bool = True
+    lens: Tuple[int, ...] = ()   # explicit prompt lengths (tests); overrides prompt_len / len_lo / len_hi
 
     @property
     def group(self) -> int:
@@ -91,6 +92,8 @@ def _seed_for(w: Workload, tag: str, layer: int = 0, step: int = 0) -> int:
 
 def seqlens(w: Workload) -> np.ndarray:
     """Prompt length of every sequence, registers included (int32 [batch])."""
+    if w.lens:
+        return np.asarray(w.lens, dtype=np.int32)
     if w.prompt_len > 0:
         return np.full((w.batch,), w.prompt_len, dtype=np.int32)
     rng = np.random.Generator(np.random.Philox(_seed_for(w, "len")))

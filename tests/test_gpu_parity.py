@@ -1,0 +1,54 @@
+"""Element-by-element parity of the CUDA library (through the C ABI) against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2507_00715_b200 import workloads as wl
+from parity_util import run_workload_and_compare
+
+pytestmark = pytest.mark.gpu
+
+BASE = wl.Workload("t", batch=3, n_layers=3, split_k=1, n_q_heads=8, n_kv_heads=2, head_dim=128, dtype="bf16",
+                   prompt_len=0, lens=(200, 77, 333), r_head=5, r_tail=3, decode_steps=3, beams=1, seed=11)
+
+
+def test_tiny_config_fp32():
+    run_workload_and_compare(wl.CONFIGS["tiny"])
+
+
+def test_bf16_ragged_gqa():
+    run_workload_and_compare(BASE)
+
+
+def test_bf16_scattered_pages():
+    run_workload_and_compare(BASE.replace(seed=12, r_head=16, r_tail=16), paged_shuffle_seed=5)
+
+
+def test_bf16_beams_group6():
+    run_workload_and_compare(BASE.replace(seed=13, n_q_heads=12, n_kv_heads=2, lens=(130, 64), batch=2, beams=3,
+                                          decode_steps=5, r_head=8, r_tail=8))
+
+
+def test_f32_head_dim_128_and_bf16_head_dim_64():
+    run_workload_and_compare(BASE.replace(seed=14, dtype="f32", lens=(65, 140), batch=2, n_q_heads=4))
+    run_workload_and_compare(BASE.replace(seed=15, head_dim=64, lens=(129, 70), batch=2))
+
+
+@pytest.mark.parametrize("rh,rt", [(0, 4), (4, 0), (0, 0), (1, 1)])
+def test_one_sided_and_no_registers(rh, rt):
+    run_workload_and_compare(BASE.replace(seed=16, r_head=rh, r_tail=rt, lens=(70, 40), batch=2))
+
+
+def test_registers_cover_whole_sequence_and_one_extra():
+    # R == L_b for the first sequence (compaction is the identity), L_b == R + 1 for the second
+    run_workload_and_compare(BASE.replace(seed=17, r_head=3, r_tail=4, lens=(7, 8, 1 + 7), batch=3))
+
+
+@pytest.mark.parametrize("k", [0, 3])
+def test_split_at_the_ends(k):
+    # k = 0: every layer is a register layer; k = N: a vanilla model that never compacts
+    run_workload_and_compare(BASE.replace(seed=18, split_k=k, lens=(90, 150), batch=2))
+
+
+def test_mha_and_many_registers():
+    run_workload_and_compare(BASE.replace(seed=19, n_q_heads=2, n_kv_heads=2, r_head=40, r_tail=37, lens=(100, 300), batch=2))
