@@ -1,0 +1,451 @@
+#!/usr/bin/env python
+"""Benchmark of the EARN attention hot path on B200.
+
+One "step" = one batch through the whole path: k full-prefill layers, N-k compaction + register
+attention layers, then T decode steps over all N layers (compact cache for l >= k, prompt cache for
+l < k).  Default workload: the 7B-class GQA configuration.  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 7b] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2507_00715_b200 import workloads as wl  # noqa: E402
+
+METRIC = "EARN attn tokens/s/GPU (prefill+decode, 7B GQA)"
+UNIT = "tokens/s"
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], tflops_burst=p["bf16_tflops"], tflops_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+def workload_desc(w: wl.Workload) -> str:
+    lens = wl.seqlens(w)
+    return (f"{w.name}: B={w.batch} N={w.n_layers} k={w.split_k} Hq/Hkv/D={w.n_q_heads}/{w.n_kv_heads}/{w.head_dim} "
+            f"{w.dtype} L={int(lens.min())}..{int(lens.max())} (sum {int(lens.sum())}) regs={w.r_head}+{w.r_tail} "
+            f"T={w.decode_steps} W={w.beams} seed={w.seed}")
+
+
+# ------------------------------------------------------------------------------------------------
+# algorithmic work (per launch) of each step of the path
+# ------------------------------------------------------------------------------------------------
+def algorithmic(w: wl.Workload):
+    lens = wl.seqlens(w).astype(np.int64)
+    es = 4 if w.dtype == "f32" else 2
+    D, Hq, Hkv, B, R, W = w.head_dim, w.n_q_heads, w.n_kv_heads, w.batch, w.n_regs, w.beams
+    tot = int(lens.sum())
+    out = {}
+    out["prefill"] = dict(flops=4.0 * D * Hq * float((lens * (lens + 1) // 2).sum()),
+                          bytes=float(tot * D * es * (2 * Hq + 2 * Hkv)))
+    out["compact"] = dict(flops=0.0, bytes=float(2 * B * R * D * es * (2 * Hkv + Hq) + B * R * 4))
+    out["register"] = dict(flops=4.0 * D * Hq * B * R * (R + 1) / 2, bytes=float(B * R * D * es * (2 * Hq + 2 * Hkv)))
+    s = w.decode_steps   # last step: the longest cache
+    qo = 2 * B * W * Hq * D * es + 4 * B * W * Hkv * D * es
+    out["decode_compact"] = dict(flops=4.0 * D * Hq * B * W * (R + s), bytes=float(2 * B * (R + W * s) * Hkv * D * es + qo))
+    out["decode_full"] = dict(flops=4.0 * D * Hq * W * (tot + B * s), bytes=float(2 * (tot + B * W * s) * Hkv * D * es + qo))
+    return out
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device: int):
+        self.proc = None
+        ident = str(device)
+        try:
+            uuid = str(torch.cuda.get_device_properties(device).uuid)
+            ident = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+        except Exception:
+            pass
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", ident, f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return None
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            text, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            return None
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in text.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return None
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+# the GPU arm
+# ------------------------------------------------------------------------------------------------
+class GpuJob:
+    def __init__(self, w: wl.Workload, device):
+        from paper_2507_00715_b200 import binding as B
+        from paper_2507_00715_b200.session import EarnSession
+        self.B = B
+        self.w = w
+        self.dev = device
+        self.ses = EarnSession(w.n_layers, w.split_k, w.n_q_heads, w.n_kv_heads, w.head_dim, w.torch_dtype,
+                               wl.cu_seqlens(w), w.r_head, w.r_tail, beams=w.beams, max_new=max(w.decode_steps, 1),
+                               device=device)
+        self.qkv = [wl.layer_qkv(w, layer, device) for layer in range(w.n_layers)]
+        self.dec = [[wl.decode_qkv(w, layer, s, device) for layer in range(w.n_layers)]
+                    for s in range(1, w.decode_steps + 1)]
+        self.parents = [None] + [torch.from_numpy(wl.beam_parents(w, s)).to(device) if w.beams > 1 else None
+                                 for s in range(2, w.decode_steps + 1)]
+        total = int(wl.cu_seqlens(w)[-1])
+        kw = dict(device=device, dtype=w.torch_dtype)
+        self.o_full = torch.empty(total, w.n_q_heads, w.head_dim, **kw)
+        self.q_reg = torch.empty(w.batch, w.n_regs, w.n_q_heads, w.head_dim, **kw)
+        self.o_reg = torch.empty_like(self.q_reg)
+        self.o_dec = torch.empty(w.batch * w.beams, w.n_q_heads, w.head_dim, **kw)
+        self.prefill_events = []
+
+    def step(self, record=False):
+        w, ses = self.w, self.ses
+        ses.lineage_cur = None
+        for layer in range(w.n_layers):
+            q, k, v = self.qkv[layer]
+            if layer < w.split_k:
+                if record:
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                ses.prefill_layer(layer, q, k, v, out=self.o_full)
+                if record:
+                    e1.record()
+                    self.prefill_events.append((e0, e1))
+            else:
+                ses.prefill_layer(layer, q, k, v, out=self.o_reg, q_reg=self.q_reg)
+        for s in range(1, w.decode_steps + 1):
+            ses.begin_step(s, self.parents[s - 1])
+            for layer in range(w.n_layers):
+                q, k, v = self.dec[s - 1][layer]
+                ses.decode_layer(layer, s, q, k, v, out=self.o_dec)
+
+    # ---- per-kernel timing in isolation (explains the step time; not the headline)
+    def time_parts(self, reps=3):
+        w, ses = self.w, self.ses
+        res = {}
+
+        def timed(fn, n_launch):
+            fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) * 1e-3 / (reps * n_launch)
+
+        early = list(range(w.split_k))
+        late = list(range(w.split_k, w.n_layers))
+        if early:
+            res["prefill"] = timed(lambda: [ses.prefill_layer(l, *self.qkv[l], out=self.o_full) for l in early], len(early))
+        if late:
+            caches = {l: ses.cache(l) for l in late}
+            res["compact"] = timed(lambda: [self.B.earn_compact_kv(ses.model, ses.batch, l, self.qkv[l][1], self.qkv[l][2],
+                                                                   caches[l], self.qkv[l][0], self.q_reg) for l in late], len(late))
+            res["register"] = timed(lambda: [self.B.earn_register_attn(ses.model, ses.batch, l, self.q_reg, caches[l],
+                                                                       self.o_reg, ses.workspace) for l in late], len(late))
+        if w.decode_steps > 0:
+            s = w.decode_steps
+            if late:
+                res["decode_compact"] = timed(lambda: [ses.decode_layer(l, s, *self.dec[s - 1][l], out=self.o_dec) for l in late], len(late))
+            if early:
+                res["decode_full"] = timed(lambda: [ses.decode_layer(l, s, *self.dec[s - 1][l], out=self.o_dec) for l in early], len(early))
+        return res
+
+    # ---- end-to-end: inputs start in pinned host memory, outputs end there
+    def setup_e2e(self):
+        def pin(t):
+            return torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
+        self.h_qkv = [tuple(pin(t) for t in trip) for trip in self.qkv]
+        self.h_dec = [[tuple(pin(t) for t in trip) for trip in row] for row in self.dec]
+        w = self.w
+        self.h_o_full = [torch.empty(self.o_full.shape, dtype=self.o_full.dtype, pin_memory=True) for _ in range(w.split_k)]
+        self.h_o_reg = [torch.empty(self.o_reg.shape, dtype=self.o_reg.dtype, pin_memory=True)
+                        for _ in range(w.n_layers - w.split_k)]
+        self.h_o_dec = torch.empty((max(w.decode_steps, 1), w.n_layers) + tuple(self.o_dec.shape), dtype=self.o_dec.dtype,
+                                   pin_memory=True)
+        nbytes = lambda t: t.numel() * t.element_size()   # noqa: E731
+        h2d = sum(nbytes(t) for trip in self.h_qkv for t in trip) + sum(nbytes(t) for row in self.h_dec for trip in row for t in trip)
+        d2h = sum(nbytes(t) for t in self.h_o_full) + sum(nbytes(t) for t in self.h_o_reg)
+        d2h += w.decode_steps * w.n_layers * nbytes(self.o_dec)
+        return h2d, d2h
+
+    def step_e2e(self):
+        w, ses = self.w, self.ses
+        ses.lineage_cur = None
+        for layer in range(w.n_layers):
+            for d, h in zip(self.qkv[layer], self.h_qkv[layer]):
+                d.copy_(h, non_blocking=True)
+            q, k, v = self.qkv[layer]
+            if layer < w.split_k:
+                ses.prefill_layer(layer, q, k, v, out=self.o_full)
+                self.h_o_full[layer].copy_(self.o_full, non_blocking=True)
+            else:
+                ses.prefill_layer(layer, q, k, v, out=self.o_reg, q_reg=self.q_reg)
+                self.h_o_reg[layer - w.split_k].copy_(self.o_reg, non_blocking=True)
+        for s in range(1, w.decode_steps + 1):
+            ses.begin_step(s, self.parents[s - 1])
+            for layer in range(w.n_layers):
+                for d, h in zip(self.dec[s - 1][layer], self.h_dec[s - 1][layer]):
+                    d.copy_(h, non_blocking=True)
+                q, k, v = self.dec[s - 1][layer]
+                ses.decode_layer(layer, s, q, k, v, out=self.o_dec)
+                self.h_o_dec[s - 1, layer].copy_(self.o_dec, non_blocking=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# the CPU oracle arm (a baseline, not a target): one sequence of the workload through every layer and step
+# ------------------------------------------------------------------------------------------------
+class OracleSample:
+    def __init__(self, w: wl.Workload, job: GpuJob | None):
+        lens = wl.seqlens(w)
+        cu = wl.cu_seqlens(w)
+        self.w1 = w.replace(batch=1, lens=(int(lens[0]),))
+        f = lambda t: t.detach().float().cpu().numpy()   # noqa: E731
+        if job is not None:       # the same tensors the GPU arm uses
+            self.qkv = [tuple(f(t[cu[0]:cu[1]]) for t in trip) for trip in job.qkv]
+            self.dec = [[tuple(f(t[:w.beams]) for t in trip) for trip in row] for row in job.dec]
+        else:                     # no device: draw the one-sequence workload on the host
+            dev = "cuda" if torch.cuda.is_available() else "cpu"
+            self.qkv = [tuple(f(t) for t in wl.layer_qkv(self.w1, l, dev)) for l in range(w.n_layers)]
+            self.dec = [[tuple(f(t) for t in wl.decode_qkv(self.w1, l, s, dev)) for l in range(w.n_layers)]
+                        for s in range(1, w.decode_steps + 1)]
+        self.parents = [None] + [wl.beam_parents(w, s)[:w.beams] if w.beams > 1 else None
+                                 for s in range(2, w.decode_steps + 1)]
+        self.tokens = int(lens[0]) + w.beams * w.decode_steps
+        self.desc = (f"sequence 0 of {w.batch} (L={int(lens[0])}, {w.beams} beam(s)): all {w.n_layers} layers of prefill "
+                     f"and all {w.decode_steps} decode steps")
+
+    def run(self) -> float:
+        from oracle import earn_oracle as orc
+        w = self.w1
+        t0 = time.perf_counter()
+        cu = np.array([0, w.lens[0]])
+        idx = orc.register_indices(w.lens, w.r_head, w.r_tail)
+        states = []
+        for layer in range(w.n_layers):
+            q, k, v = self.qkv[layer]
+            if layer < w.split_k:
+                orc.causal_attention(q, k, v, cu)
+                states.append(orc.DecodeState([k], [v], w.beams))
+            else:
+                kc, vc, qc = orc.compact(k, cu, idx), orc.compact(v, cu, idx), orc.compact(q, cu, idx)
+                orc.register_attention(qc, kc, vc)
+                states.append(orc.DecodeState([kc[0]], [vc[0]], w.beams))
+        for s in range(1, w.decode_steps + 1):
+            for layer in range(w.n_layers):
+                q, k, v = self.dec[s - 1][layer]
+                states[layer].step(q, k, v, self.parents[s - 1])
+        return time.perf_counter() - t0
+
+
+def blas_threads() -> int:
+    try:
+        import threadpoolctl
+        return max([p["num_threads"] for p in threadpoolctl.threadpool_info() if p.get("user_api") == "blas"] or [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+# ------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="7b", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--split-k", type=int, default=None)
+    ap.add_argument("--impl", default="earn", choices=["earn", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-parts", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "earn" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    w = wl.CONFIGS[args.config]
+    if args.split_k is not None:
+        w = w.replace(split_k=args.split_k)
+    lens = wl.seqlens(w)
+    tokens_per_step = int(lens.sum()) + w.batch * w.beams * w.decode_steps
+    config = {"workload": workload_desc(w), "l2": "per-layer inputs and caches exceed the 126 MB L2; no flush needed",
+              "sharding": "every rank runs the whole batch of its own seed (no data-path collective)"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        sample = OracleSample(w, None)
+        for _ in range(args.warmup):
+            sample.run()
+        times = [sample.run() for _ in range(args.steps)]
+        t = sum(times) / len(times)
+        val = sample.tokens / t
+        print(json.dumps({
+            "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": config,
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample.desc},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        return
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    import __graft_entry__ as entry
+    if local_rank == 0:
+        entry.build()
+    if dist is not None:
+        dist.barrier()
+    from paper_2507_00715_b200 import binding as B
+
+    job = GpuJob(w.replace(seed=w.seed + 1000 * rank) if rank else w, dev)
+    peaks = read_peaks()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        job.step()
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    n0 = B.earn_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        job.step(record=True)
+    e1.record()
+    barrier()
+    launches = B.earn_launch_count() - n0
+    clocks = sampler.stop() if sampler else None
+    elapsed = e0.elapsed_time(e1) * 1e-3
+    if dist is not None:
+        t = torch.tensor([elapsed], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed = float(t.item())
+    assert job.ses.device_status() == 0, "a device-side wait timed out"
+    t_step = elapsed / args.steps
+    value = world * tokens_per_step / t_step
+
+    # roofline of the dominant kernel (prefill), from the events recorded inside the timed region
+    alg = algorithmic(w)
+    roofline = None
+    if job.prefill_events:
+        t_pre = sum(a.elapsed_time(b) for a, b in job.prefill_events) * 1e-3 / len(job.prefill_events)
+        ach = alg["prefill"]["flops"] / t_pre / 1e12
+        roofline = {"kernel": "earn_prefill_attn", "bound": "tensor", "achieved": ach, "peak": peaks["tflops_sustained"],
+                    "unit": "TFLOP/s", "frac": ach / peaks["tflops_sustained"], "peak_source": peaks["source"] + " (sustained)",
+                    "traffic": None, "avg_launch_ms": t_pre * 1e3, "launches": len(job.prefill_events),
+                    "share_of_step": t_pre * w.split_k / t_step,
+                    "algorithmic_flops_per_launch": alg["prefill"]["flops"], "algorithmic_bytes_per_launch": alg["prefill"]["bytes"]}
+
+    parts = None
+    if not args.no_parts and rank == 0:
+        tp = job.time_parts()
+        parts = {}
+        for name, sec in tp.items():
+            a = alg[name]
+            parts[name] = {"ms_per_launch": sec * 1e3, "GB_s": a["bytes"] / sec / 1e9, "hbm_frac": a["bytes"] / sec / 1e9 / peaks["hbm_gbs"],
+                           "TFLOP_s": a["flops"] / sec / 1e12, "tensor_frac": a["flops"] / sec / 1e12 / peaks["tflops_burst"]}
+
+    e2e = None
+    if not args.no_e2e:
+        h2d, d2h = job.setup_e2e()
+        job.step_e2e()
+        barrier()
+        n_e2e = max(1, min(args.steps, 2))
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for _ in range(n_e2e):
+            job.step_e2e()
+        a1.record()
+        barrier()
+        te = a0.elapsed_time(a1) * 1e-3 / n_e2e
+        if dist is not None:
+            t = torch.tensor([te], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            te = float(t.item())
+        e2e = {"value": world * tokens_per_step / te, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": te * 1e3, "steps": n_e2e}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sample = OracleSample(w, job)
+        tc = sample.run()
+        cpu = {"value": sample.tokens / tc, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample.desc,
+               "seconds": tc}
+
+    if rank == 0:
+        T, N, k = w.decode_steps, w.n_layers, w.split_k
+        extra = {}
+        if parts:
+            t_prefill = k * parts.get("prefill", {}).get("ms_per_launch", 0) + (N - k) * (
+                parts.get("compact", {}).get("ms_per_launch", 0) + parts.get("register", {}).get("ms_per_launch", 0))
+            extra["prefill_tokens_per_s_isolated"] = int(lens.sum()) / (t_prefill * 1e-3) if t_prefill else None
+        earn_e, van_e = job.ses.kv_entries(T), N * (int(lens.sum()) + w.batch * w.beams * T)
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": w.dtype, "data": "synthetic", "config": config, "clocks": clocks, "e2e": e2e,
+            "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
+            "sequences_per_s": world * w.batch / t_step, "kernels": parts, "kv_reduction": 1.0 - earn_e / van_e,
+            "peaks": peaks, **extra}))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -151,6 +151,9 @@ earn_status_t earn_beam_reparent(int32_t batch, int32_t beams, int32_t max_new, 
                                  const int32_t* parent, const int32_t* lineage_in_or_null,
                                  int32_t* lineage_out, earn_stream_t stream);
 
+/* Number of kernels this library has launched in this process so far (host counter, all streams). */
+uint64_t earn_launch_count(void);
+
 const char* earn_status_string(earn_status_t status);
 int32_t earn_version(void);
 

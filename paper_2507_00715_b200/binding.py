@@ -57,6 +57,7 @@ SYMBOLS = {
                                    C.c_void_p, C.c_size_t, C.c_void_p]),
     "earn_beam_reparent": (C.c_int, [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.c_void_p]),
+    "earn_launch_count": (C.c_uint64, []),
     "earn_status_string": (C.c_char_p, [C.c_int]),
     "earn_version": (C.c_int32, []),
 }
@@ -139,6 +140,10 @@ def make_cache(k_shared=None, v_shared=None, block_table=None, pages_per_seq=0, 
 
 def earn_version() -> int:
     return lib().earn_version()
+
+
+def earn_launch_count() -> int:
+    return int(lib().earn_launch_count())
 
 
 def earn_workspace_bytes(model: EarnModel, batch: Batch, beams: int) -> int:

@@ -227,6 +227,7 @@ cudaError_t launch_one(const SimtParams& p, dim3 grid, cudaStream_t st) {
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   kern<<<grid, 256, smem, st>>>(p);
+  note_launch();
   return cudaGetLastError();
 }
 
@@ -364,6 +365,7 @@ cudaError_t launch_decode_simt(const DecodeArgs& a, cudaStream_t st) {
     if (e != cudaSuccess) return e;
   }
   dim3 grid((a.Hq + 3) / 4, a.batch * a.beams);
+  note_launch();
   if (a.dtype == EARN_F32) {
     if (a.D == 64) decode_merge_kernel<float, 64><<<grid, 128, 0, st>>>(a);
     else decode_merge_kernel<float, 128><<<grid, 128, 0, st>>>(a);

@@ -56,12 +56,14 @@ __global__ void beam_reparent_kernel(int beams, int max_new, int step, const int
 cudaError_t launch_compact(const CompactArgs& a, cudaStream_t st) {
   dim3 grid(a.r_head + a.r_tail, a.batch);
   compact_kernel<<<grid, 128, 0, st>>>(a);
+  note_launch();
   return cudaGetLastError();
 }
 
 cudaError_t launch_beam_reparent(int batch, int beams, int max_new, int step, const int32_t* parent,
                                  const int32_t* lineage_in, int32_t* lineage_out, cudaStream_t st) {
   int n = batch * beams * max_new;
+  note_launch();
   beam_reparent_kernel<<<(n + 255) / 256, 256, 0, st>>>(beams, max_new, step, parent, lineage_in, lineage_out,
                                                         batch * beams);
   return cudaGetLastError();

@@ -1,10 +1,14 @@
 // C-ABI entry points: host-side validation, workspace layout and kernel dispatch.
 #include <cstdio>
 #include <cstring>
+#include <atomic>
 
 #include "earn_common.cuh"
 
 namespace earn {
+
+static std::atomic<uint64_t> g_launches{0};
+void note_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -104,6 +108,8 @@ using namespace earn;
 extern "C" {
 
 int32_t earn_version(void) { return 100; }
+
+uint64_t earn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* earn_status_string(earn_status_t s) {
   switch (s) {

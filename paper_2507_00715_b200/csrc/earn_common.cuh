@@ -46,6 +46,8 @@ constexpr int kDecodeRows = 16;
 DecodePlan make_decode_plan(const earn_model_t& m, const earn_batch_t& b, int beams, int max_shared_len);
 size_t decode_partial_floats(const earn_model_t& m, const earn_batch_t& b, const DecodePlan& p);
 
+void note_launch(int n = 1);   // host-side count of kernels launched by this library
+
 // ---- launchers (one per .cu file); all return cudaGetLastError() of their launches ----
 struct PrefillArgs {
   const void *q, *k, *v;
