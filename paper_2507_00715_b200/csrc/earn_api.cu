@@ -160,6 +160,11 @@ earn_status_t earn_prefill_attn(const earn_model_t* model, const earn_batch_t* b
   a.batch = batch->batch; a.max_seqlen = batch->max_seqlen;
   a.Hq = model->n_q_heads; a.Hkv = model->n_kv_heads; a.D = model->head_dim; a.dtype = model->dtype;
   a.scale = scale_of(model);
+  if (prefill_tc_supported(a, batch->total_tokens)) {
+    if (!aligned16(workspace)) return EARN_ERR_WORKSPACE;
+    return launch_prefill_tc(a, batch->total_tokens, reinterpret_cast<int32_t*>(workspace), (cudaStream_t)stream) ==
+                   cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+  }
   return launch_prefill_simt(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
 }
 

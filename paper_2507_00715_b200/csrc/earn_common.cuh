@@ -58,6 +58,9 @@ struct PrefillArgs {
   float scale;
 };
 cudaError_t launch_prefill_simt(const PrefillArgs& a, cudaStream_t st);
+// tensor-core path (bf16, head_dim 128); status_word receives EARN_ERR_TIMEOUT if a bounded wait runs out
+bool prefill_tc_supported(const PrefillArgs& a, int total_tokens);
+cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int32_t* status_word, cudaStream_t st);
 
 struct RegisterArgs {
   const void* q_reg;
