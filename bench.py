@@ -285,6 +285,43 @@ class OracleSample:
         return time.perf_counter() - t0
 
 
+def profile_one_kernel(w: wl.Workload, dev, which: str, launches: int = 3):
+    """One layer of the workload, one kind of launch, `launches` times (a few GB at most on the device)."""
+    early = which in ("prefill", "decode_full")
+    # keep the layer on the side of the split the kernel belongs to; one full layer + one register layer
+    w1 = w.replace(n_layers=2, split_k=1)
+    layer = 0 if early else 1
+    job = GpuJob.__new__(GpuJob)
+    from paper_2507_00715_b200 import binding as B
+    from paper_2507_00715_b200.session import EarnSession
+    ses = EarnSession(w1.n_layers, w1.split_k, w1.n_q_heads, w1.n_kv_heads, w1.head_dim, w1.torch_dtype,
+                      wl.cu_seqlens(w1), w1.r_head, w1.r_tail, beams=w1.beams, max_new=max(w1.decode_steps, 1), device=dev)
+    q, k, v = wl.layer_qkv(w1, layer, dev)
+    o = torch.empty_like(q)
+    q_reg = torch.empty(w1.batch, w1.n_regs, w1.n_q_heads, w1.head_dim, device=dev, dtype=w1.torch_dtype)
+    o_reg = torch.empty_like(q_reg)
+    s_last = max(w1.decode_steps, 1)
+    dq, dk, dv = wl.decode_qkv(w1, layer, s_last, dev)
+    o_dec = torch.empty_like(dq)
+    if early:
+        ses.prefill_layer(0, q, k, v, out=o)            # also registers the prompt K/V for decode
+    else:
+        ses.prefill_layer(1, q, k, v, out=o_reg, q_reg=q_reg)
+    torch.cuda.synchronize()
+    for _ in range(launches):
+        if which == "prefill":
+            ses.prefill_layer(0, q, k, v, out=o)
+        elif which == "compact":
+            B.earn_compact_kv(ses.model, ses.batch, 1, k, v, ses.cache(1), q, q_reg)
+        elif which == "register":
+            B.earn_register_attn(ses.model, ses.batch, 1, q_reg, ses.cache(1), o_reg, ses.workspace)
+        else:
+            ses.decode_layer(layer, s_last, dq, dk, dv, out=o_dec)
+    torch.cuda.synchronize()
+    assert ses.device_status() == 0
+    print(json.dumps({"profiled": which, "workload": workload_desc(w1), "launches": launches}))
+
+
 def blas_threads() -> int:
     try:
         import threadpoolctl
@@ -305,6 +342,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-parts", action="store_true")
+    ap.add_argument("--profile-kernel", default=None,
+                    choices=["prefill", "compact", "register", "decode_compact", "decode_full"],
+                    help="small case for a profiler: allocate ONE layer of the workload and launch that step 3 times")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "earn" else args.warmup
 
@@ -349,6 +389,10 @@ def main():
     if dist is not None:
         dist.barrier()
     from paper_2507_00715_b200 import binding as B
+
+    if args.profile_kernel:
+        profile_one_kernel(w, dev, args.profile_kernel)
+        return
 
     job = GpuJob(w.replace(seed=w.seed + 1000 * rank) if rank else w, dev)
     peaks = read_peaks()
