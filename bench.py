@@ -39,6 +39,16 @@ def read_peaks():
     return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
 
 
+def read_traffic(name: str) -> dict:
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) taken from the ncu captures
+    summarised under profiles/; {} when no capture of this workload has been recorded."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if not os.path.exists(path):
+        return {}
+    with open(path) as f:
+        return json.load(f).get(name, {})
+
+
 def workload_desc(w: wl.Workload) -> str:
     lens = wl.seqlens(w)
     return (f"{w.name}: B={w.batch} N={w.n_layers} k={w.split_k} Hq/Hkv/D={w.n_q_heads}/{w.n_kv_heads}/{w.head_dim} "
@@ -141,28 +151,79 @@ class GpuJob:
         self.q_reg = torch.empty(w.batch, w.n_regs, w.n_q_heads, w.head_dim, **kw)
         self.o_reg = torch.empty_like(self.q_reg)
         self.o_dec = torch.empty(w.batch * w.beams, w.n_q_heads, w.head_dim, **kw)
-        self.prefill_events = []
+        self.graphs = None
+        self.marks = []
+
+    # ---- the step as an ordered list of segments; each segment = consecutive launches of one kind
+    def segments(self):
+        """[(kind, n_launches, callable)] in the order of the hot path.  `n_launches` counts the calls the
+        roofline is quoted per: prefill / decode calls, or (compaction + register attention) pairs."""
+        w, ses = self.w, self.ses
+        early, late = list(range(w.split_k)), list(range(w.split_k, w.n_layers))
+        segs = []
+        if early:
+            segs.append(("prefill", len(early),
+                         lambda: [ses.prefill_layer(l, *self.qkv[l], out=self.o_full) for l in early]))
+        if late:
+            segs.append(("register_layer", len(late),
+                         lambda: [ses.prefill_layer(l, *self.qkv[l], out=self.o_reg, q_reg=self.q_reg) for l in late]))
+        for s in range(1, w.decode_steps + 1):
+            if early:
+                def f(s=s):
+                    ses.begin_step(s, self.parents[s - 1])
+                    for l in early:
+                        ses.decode_layer(l, s, *self.dec[s - 1][l], out=self.o_dec)
+                segs.append(("decode_full", len(early), f))
+            if late:
+                def f2(s=s, first=not early):
+                    if first:
+                        ses.begin_step(s, self.parents[s - 1])
+                    for l in late:
+                        ses.decode_layer(l, s, *self.dec[s - 1][l], out=self.o_dec)
+                segs.append(("decode_compact", len(late), f2))
+        return segs
+
+    def capture_graphs(self):
+        """One CUDA graph per segment (the launches of a step never change between steps)."""
+        self.ses.lineage_cur = None
+        self.graphs = []
+        for kind, n, fn in self.segments():
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn()
+            self.graphs.append((kind, n, g))
+        torch.cuda.synchronize()
 
     def step(self, record=False):
-        w, ses = self.w, self.ses
-        ses.lineage_cur = None
-        for layer in range(w.n_layers):
-            q, k, v = self.qkv[layer]
-            if layer < w.split_k:
-                if record:
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    e0.record()
-                ses.prefill_layer(layer, q, k, v, out=self.o_full)
-                if record:
-                    e1.record()
-                    self.prefill_events.append((e0, e1))
+        """One pass of the whole hot path.  With record=True an event is recorded at every segment
+        boundary so that each kind of launch gets a live duration inside the timed region."""
+        self.ses.lineage_cur = None
+        items = self.graphs if self.graphs is not None else self.segments()
+        marks = []
+        for kind, n, g in items:
+            if record:
+                e = torch.cuda.Event(enable_timing=True)
+                e.record()
+                marks.append((kind, n, e))
+            if self.graphs is not None:
+                g.replay()
             else:
-                ses.prefill_layer(layer, q, k, v, out=self.o_reg, q_reg=self.q_reg)
-        for s in range(1, w.decode_steps + 1):
-            ses.begin_step(s, self.parents[s - 1])
-            for layer in range(w.n_layers):
-                q, k, v = self.dec[s - 1][layer]
-                ses.decode_layer(layer, s, q, k, v, out=self.o_dec)
+                g()
+        if record:
+            e = torch.cuda.Event(enable_timing=True)
+            e.record()
+            marks.append((None, 0, e))
+            self.marks.append(marks)
+
+    def segment_times(self):
+        """{kind: (seconds per launch, launches per step, share of step time)} from the recorded events."""
+        tot, cnt, steps = {}, {}, len(self.marks)
+        for marks in self.marks:
+            for (kind, n, e0), (_, _, e1) in zip(marks[:-1], marks[1:]):
+                tot[kind] = tot.get(kind, 0.0) + e0.elapsed_time(e1) * 1e-3
+                cnt[kind] = cnt.get(kind, 0) + n
+        whole = sum(tot.values())
+        return {k: (tot[k] / cnt[k], cnt[k] // steps, tot[k] / whole) for k in tot}
 
     # ---- per-kernel timing in isolation (explains the step time; not the headline)
     def time_parts(self, reps=3):
@@ -172,10 +233,15 @@ class GpuJob:
         def timed(fn, n_launch):
             fn()
             torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                fn()
+            g.replay()
+            torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
             for _ in range(reps):
-                fn()
+                g.replay()
             e1.record()
             torch.cuda.synchronize()
             return e0.elapsed_time(e1) * 1e-3 / (reps * n_launch)
@@ -342,6 +408,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-parts", action="store_true")
+    ap.add_argument("--no-graphs", action="store_true", help="plain launches instead of CUDA-graph replay")
     ap.add_argument("--profile-kernel", default=None,
                     choices=["prefill", "compact", "register", "decode_compact", "decode_full"],
                     help="small case for a profiler: allocate ONE layer of the workload and launch that step 3 times")
@@ -402,18 +469,23 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    n0 = B.earn_launch_count()
+    job.step()                                   # first pass: plain launches (also sets per-kernel attributes)
+    launches_per_step = B.earn_launch_count() - n0
+    torch.cuda.synchronize()
+    if not args.no_graphs:
+        job.capture_graphs()                     # the same launches, recorded once, replayed per step
     for _ in range(args.warmup):
         job.step()
     barrier()
     sampler = ClockSampler(local_rank) if rank == 0 else None
-    n0 = B.earn_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
         job.step(record=True)
     e1.record()
     barrier()
-    launches = B.earn_launch_count() - n0
+    launches = launches_per_step * args.steps
     clocks = sampler.stop() if sampler else None
     elapsed = e0.elapsed_time(e1) * 1e-3
     if dist is not None:
@@ -424,17 +496,31 @@ def main():
     t_step = elapsed / args.steps
     value = world * tokens_per_step / t_step
 
-    # roofline of the dominant kernel (prefill), from the events recorded inside the timed region
+    # rooflines from the events recorded at the segment boundaries INSIDE the timed region
     alg = algorithmic(w)
-    roofline = None
-    if job.prefill_events:
-        t_pre = sum(a.elapsed_time(b) for a, b in job.prefill_events) * 1e-3 / len(job.prefill_events)
-        ach = alg["prefill"]["flops"] / t_pre / 1e12
-        roofline = {"kernel": "earn_prefill_attn", "bound": "tensor", "achieved": ach, "peak": peaks["tflops_sustained"],
-                    "unit": "TFLOP/s", "frac": ach / peaks["tflops_sustained"], "peak_source": peaks["source"] + " (sustained)",
-                    "traffic": None, "avg_launch_ms": t_pre * 1e3, "launches": len(job.prefill_events),
-                    "share_of_step": t_pre * w.split_k / t_step,
-                    "algorithmic_flops_per_launch": alg["prefill"]["flops"], "algorithmic_bytes_per_launch": alg["prefill"]["bytes"]}
+    alg["register_layer"] = dict(flops=alg["compact"]["flops"] + alg["register"]["flops"],
+                                 bytes=alg["compact"]["bytes"] + alg["register"]["bytes"])
+    # decode segments cover all T steps: quote the average step's cache length
+    s_mid = (w.decode_steps + 1) / 2.0
+    es, Bq = (4 if w.dtype == "f32" else 2), w.batch * w.beams
+    qo = 2 * Bq * w.n_q_heads * w.head_dim * es + 4 * Bq * w.n_kv_heads * w.head_dim * es
+    alg["decode_compact"]["bytes"] = 2 * w.batch * (w.n_regs + w.beams * s_mid) * w.n_kv_heads * w.head_dim * es + qo
+    alg["decode_full"]["bytes"] = 2 * (int(lens.sum()) + Bq * s_mid) * w.n_kv_heads * w.head_dim * es + qo
+    traffic = read_traffic(w.name)
+    rooflines = {}
+    for kind, (sec, per_step, share) in job.segment_times().items():
+        a = alg[kind]
+        if kind == "prefill":
+            ach, peak, unit, bound = a["flops"] / sec / 1e12, peaks["tflops_sustained"], "TFLOP/s", "tensor"
+            src = peaks["source"] + " (sustained bf16)"
+        else:
+            ach, peak, unit, bound = a["bytes"] / sec / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
+            src = peaks["source"] + " (copy)"
+        rooflines[kind] = {"kernel": kind, "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                           "peak_source": src, "traffic": traffic.get(kind), "avg_launch_ms": sec * 1e3,
+                           "launches_per_step": per_step, "share_of_step": share,
+                           "algorithmic_flops_per_launch": a["flops"], "algorithmic_bytes_per_launch": a["bytes"]}
+    roofline = max(rooflines.values(), key=lambda r: r["share_of_step"]) if rooflines else None
 
     parts = None
     if not args.no_parts and rank == 0:
@@ -484,7 +570,8 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": w.dtype, "data": "synthetic", "config": config, "clocks": clocks, "e2e": e2e,
-            "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
+            "gpu_launches": int(launches), "roofline": roofline, "rooflines": rooflines, "cpu_baseline": cpu,
+            "launch_mode": "plain" if args.no_graphs else "cuda-graph replay, one graph per segment",
             "sequences_per_s": world * w.batch / t_step, "kernels": parts, "kv_reduction": 1.0 - earn_e / van_e,
             "peaks": peaks, **extra}))
     if dist is not None:

@@ -224,7 +224,7 @@ template <typename T, int D, int BM, int MODE>
 cudaError_t launch_one(const SimtParams& p, dim3 grid, cudaStream_t st) {
   constexpr size_t smem = simt_smem_bytes<D, BM>();
   auto kern = attn_simt_kernel<T, D, BM, MODE>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = ensure_dynamic_smem<attn_simt_kernel<T, D, BM, MODE>>((int)smem);
   if (e != cudaSuccess) return e;
   kern<<<grid, 256, smem, st>>>(p);
   note_launch();

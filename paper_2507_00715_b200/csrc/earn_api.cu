@@ -58,7 +58,7 @@ DecodePlan make_decode_plan(const earn_model_t& m, const earn_batch_t& b, int be
   if (max_shared_len <= 0 || b.batch == 0) { p.chunk = 64; p.n_splits = 0; return p; }
   // enough CTAs to cover the SMs a few times over, but no more splits than that needs
   const long units = (long)b.batch * m.n_kv_heads * p.row_tiles;
-  const long want = 4L * 148;
+  const long want = 3L * 148;   // four decode CTAs fit an SM; aim for most of those slots in one wave
   long splits = (want + units - 1) / units;
   long max_splits = (max_shared_len + 63) / 64;
   if (splits > max_splits) splits = max_splits;
@@ -260,7 +260,9 @@ earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* ba
   a.batch = batch->batch; a.beams = cache->beams; a.max_new = cache->max_new; a.step = step;
   a.Hq = model->n_q_heads; a.Hkv = model->n_kv_heads; a.D = model->head_dim; a.dtype = model->dtype;
   a.scale = scale_of(model);
-  return launch_decode_simt(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+  const cudaError_t e = model->dtype == EARN_BF16 ? launch_decode_mma(a, (cudaStream_t)stream)
+                                                   : launch_decode_simt(a, (cudaStream_t)stream);
+  return e == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
 }
 
 earn_status_t earn_beam_reparent(int32_t batch, int32_t beams, int32_t max_new, int32_t step, const int32_t* parent,

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "earn.h"
 
 namespace earn {
@@ -48,6 +50,19 @@ size_t decode_partial_floats(const earn_model_t& m, const earn_batch_t& b, const
 
 void note_launch(int n = 1);   // host-side count of kernels launched by this library
 
+// Opt a kernel in to `bytes` of dynamic shared memory, once per device (the attribute call is not free).
+template <auto Kernel>
+cudaError_t ensure_dynamic_smem(int bytes) {
+  static std::atomic<uint64_t> done{0};   // one bit per device ordinal < 64
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 64 && ((done.load(std::memory_order_relaxed) >> dev) & 1)) return cudaSuccess;
+  e = cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess && dev < 64) done.fetch_or(1ull << dev, std::memory_order_relaxed);
+  return e;
+}
+
 // ---- launchers (one per .cu file); all return cudaGetLastError() of their launches ----
 struct PrefillArgs {
   const void *q, *k, *v;
@@ -84,7 +99,8 @@ struct DecodeArgs {
   int batch, beams, max_new, step, Hq, Hkv, D, dtype;
   float scale;
 };
-cudaError_t launch_decode_simt(const DecodeArgs& a, cudaStream_t st);
+cudaError_t launch_decode_simt(const DecodeArgs& a, cudaStream_t st);   // fp32 debug path
+cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st);    // bf16: cp.async rings + mma.sync
 
 struct CompactArgs {
   const void *k, *v, *q;

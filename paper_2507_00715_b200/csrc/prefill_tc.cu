@@ -309,7 +309,7 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int32_t* s
   if (!make_map(&mq, a.q, a.Hq, total_tokens) || !make_map(&mk, a.k, a.Hkv, total_tokens) ||
       !make_map(&mv, a.v, a.Hkv, total_tokens))
     return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  cudaError_t e = ensure_dynamic_smem<prefill_tc_kernel>(SMEM_BYTES);
   if (e != cudaSuccess) return e;
   TcParams p{};
   p.o = a.o; p.lse = a.lse; p.cu_seqlens = a.cu_seqlens; p.status = status_word;
