@@ -95,7 +95,9 @@ typedef struct {
  * width (0 is never returned; the first 256 bytes hold the device status word).  Host only. */
 size_t earn_workspace_bytes(const earn_model_t* model, const earn_batch_t* batch, int32_t beams);
 
-/* Clears the device status word.  Call once after allocating the workspace (asynchronous). */
+/* Zeroes the workspace: the device status word and the split-decode tickets must start at zero.  Call once
+ * after allocating the workspace and before the first call that uses it (asynchronous on `stream`).  A
+ * workspace is used by one stream at a time: calls that overlap on the GPU must not share one. */
 earn_status_t earn_workspace_init(void* workspace, size_t workspace_bytes, earn_stream_t stream);
 
 /* Synchronises `stream` and returns the device status word of the workspace: EARN_OK, or

@@ -1,68 +1,64 @@
 // Decode attention (Eq. 4: append K_t, V_t, then attend over K_{1:t}) for bf16 caches.
 //
 // HBM-bound: every byte of the cache is read once per step, so the kernel is built around keeping
-// enough loads in flight, not around the tensor cores; warp-level mma.sync (m16n8k16) only keeps the
-// few query rows per key (g heads x W beams, padded to 16) off the FMA pipe.
+// loads in flight with few instructions, not around the tensor cores; warp-level mma.sync (m16n8k16)
+// only keeps the few query rows per key (g heads x W beams, padded to 16) off the FMA pipe.
 //
-// One CTA = (sequence b, kv head, split of the shared segment, tile of 16 query rows); 2 warps.  The key
+// One CTA = (sequence b, kv head, split of the shared segment, tile of 16 query rows); 1 warp.  The key
 // list of a CTA is its chunk of the shared segment (the prompt K/V of a layer l < k read in place, or
 // the compact register pages of a layer l >= k) followed -- in split 0 only -- by the generated tokens
 // of the beams its rows belong to (masked per row to the row's own beam; the newest token comes
-// straight from k_new / v_new, which split 0 also appends to the private segment).  Tiles of 16 keys are
-// dealt round-robin to the warps; each warp runs its own 3-stage cp.async ring (no block-wide barrier
-// in the main loop) and an online softmax in the log2 domain.  The per-warp partial results are merged
-// through shared memory.  With a single split the CTA writes O itself; otherwise it writes a normalised
-// partial + log2-domain LSE and decode_combine_kernel folds the splits.
+// straight from k_new / v_new, which split 0 also appends to the private segment).
+//
+// The list is cut into tiles of 16 positions.  The warp fetches them with 16-byte cp.async copies into
+// padded shared-memory tiles (a ring of four stages = 35 KB at head_dim 128, so six CTAs share an SM; two
+// stages for lists of at most two tiles).  Tile size, warps per CTA and ring depth were swept on B200 at
+// the 7B shapes: (16, 1, 4) gave 50.9 us per layer against 51.3-63.4 us for the other combinations.
+// Rows that are an affine function of the list position (packed prompt K/V, identity page table)
+// take a fast path of pointer increments; any other tile (scattered pages, generated tokens
+// behind the lineage table, a ragged last tile) first resolves one row per lane and hands the row
+// offsets to the copying lanes by shuffle.  (One bulk copy per 256-byte row measured 4.0 TB/s on B200
+// against 6.2 TB/s for this scheme: the row is too small a unit for the copy engine.)
+// Online softmax in the log2 domain.  With a single split the CTA writes O itself; otherwise it writes a
+// normalised partial + log2-domain LSE, takes a ticket, and the CTA holding the last ticket of its
+// (sequence, kv head, row tile) folds the partials -- one launch, and no CTA ever waits for another.
 #include "earn_common.cuh"
+#include "mma_sync.cuh"
+#include "sm100_ptx.cuh"
 
 namespace earn {
 namespace {
+using namespace mma;
 
-constexpr int KT = 16;       // keys per tile
-constexpr int STAGES = 3;    // cp.async ring depth per warp
-constexpr int NWARPS = 2;    // 48 KB of rings per CTA at head_dim 128: four CTAs share an SM
+#ifndef EARN_DECODE_KT
+#define EARN_DECODE_KT 16
+#endif
+#ifndef EARN_DECODE_NWARPS
+#define EARN_DECODE_NWARPS 1
+#endif
+#ifndef EARN_DECODE_STAGES
+#define EARN_DECODE_STAGES 4
+#endif
+constexpr int KT = EARN_DECODE_KT;           // list positions per tile (16 or 32)
+constexpr int NWARPS = EARN_DECODE_NWARPS;   // warps per CTA; tiles are dealt round-robin to them
+constexpr int N8 = KT / 8, H16 = KT / 16;
 
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+template <int D, int STAGES>   // STAGES: cp.async ring depth per warp
+struct Geo {
+  static constexpr int ROWB = D * 2;            // bytes of one K (or V) row
+  static constexpr int PITCH = ROWB + 16;       // padded row pitch: conflict-free ldmatrix, 16-byte aligned
+  static constexpr int TILE_B = KT * PITCH;     // one K (or V) tile
+  static constexpr int STAGE_B = 2 * TILE_B;    // K tile + V tile
+  static constexpr int RING_B = NWARPS * STAGES * STAGE_B;
+  static constexpr int MERGE_B = NWARPS * 16 * D * 4 + NWARPS * 16 * 2 * 4 + 16;
+  static constexpr int DATA_B = RING_B > MERGE_B ? RING_B : MERGE_B;
+  static constexpr int SMEM_B = DATA_B;
+};
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&t);
-}
-
-template <int D>
-constexpr int decode_smem_bytes() {
-  // the cp.async rings; reused for the cross-warp merge (NWARPS x 16 x D fp32 + statistics)
-  constexpr int ring = NWARPS * STAGES * 2 * KT * D * 2;
-  constexpr int merge = NWARPS * 16 * D * 4 + NWARPS * 16 * 2 * 4;
-  return ring > merge ? ring : merge;
-}
-
-template <int D>
+template <int D, int STAGES>
 __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   using bf16 = __nv_bfloat16;
-  constexpr int ROWB = D * 2;          // bytes per key row
-  constexpr int CH = ROWB / 16;        // 16-byte chunks per row
-  constexpr int TILE_B = KT * ROWB;    // bytes of one K (or V) tile
+  using G = Geo<D, STAGES>;
   constexpr int KSTEPS = D / 16, NTILES = D / 8;
   extern __shared__ __align__(128) uint8_t smem[];
 
@@ -71,14 +67,15 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   const int row_tiles = a.plan.row_tiles;
   const int split = blockIdx.x / row_tiles, row0 = (blockIdx.x % row_tiles) * 16;
   const int g = a.Hq / a.Hkv, W = a.beams, n_rows = W * g, step = a.step;
-  const int shared_len = a.src.paged ? a.src.n_regs : (a.cu_seqlens[b + 1] - a.cu_seqlens[b]);
+  const int seq_lo = a.src.paged ? 0 : a.cu_seqlens[b];
+  const int shared_len = a.src.paged ? a.src.n_regs : (a.cu_seqlens[b + 1] - seq_lo);
   const int key_begin = split * a.plan.chunk;
-  const int key_end = min(key_begin + a.plan.chunk, shared_len);
-  const int n_shared = max(key_end - key_begin, 0);
+  const int n_shared = max(min(key_begin + a.plan.chunk, shared_len) - key_begin, 0);
   const int w_lo = row0 / g, w_hi = min((row0 + 15) / g, W - 1);
   const int n_priv = (split == 0) ? (w_hi - w_lo + 1) * step : 0;
-  if (n_shared == 0 && n_priv == 0) return;
-  const int tiles_sh = (n_shared + KT - 1) / KT, n_tiles = tiles_sh + (n_priv + KT - 1) / KT;
+  const int n_total = n_shared + n_priv;
+  if (n_total == 0) return;
+  const int n_tiles = (n_total + KT - 1) / KT;
   const float scale_log2 = a.scale * kLog2e;
 
   const bf16* kg = reinterpret_cast<const bf16*>(a.src.k);
@@ -88,8 +85,72 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   const bf16* kn = reinterpret_cast<const bf16*>(a.k_new);
   const bf16* vn = reinterpret_cast<const bf16*>(a.v_new);
 
+  // ---- per-warp cp.async ring.  A copy instruction moves 32 x 16 bytes = RPI whole rows.
+  constexpr int CH = G::ROWB / 16, RPI = 32 / CH, NIT = KT / RPI;
+  const uint32_t ring = ptx::smem_u32(smem) + warp * (STAGES * G::STAGE_B);
+  const int ch = lane % CH, r0 = lane / CH;
+  const uint32_t dst0 = (uint32_t)r0 * G::PITCH + (uint32_t)ch * 16;
+  const int64_t rowstride = (int64_t)a.Hkv * D;   // elements between consecutive rows of a tensor
+  // shared rows that are affine in the list position: row(p) = row_base + key_begin + p
+  const bool affine = !a.src.paged || a.src.block_table == nullptr;
+  const int64_t row_base = a.src.paged ? (int64_t)b * a.src.pages_per_seq * EARN_PAGE_TOKENS : (int64_t)seq_lo;
+  const int64_t fast_off = ((row_base + key_begin + r0) * a.Hkv + kvh) * D + ch * 8;
+
+  auto issue_tile = [&](int tile, int stage) {
+    const uint32_t kdst = ring + stage * G::STAGE_B + dst0, vdst = kdst + G::TILE_B;
+    if (affine && (tile + 1) * KT <= n_shared) {
+      const bf16* ks = kg + fast_off + (int64_t)tile * KT * rowstride;
+      const bf16* vs = vg + fast_off + (int64_t)tile * KT * rowstride;
+#pragma unroll
+      for (int i = 0; i < NIT; ++i) {
+        cp_async16(kdst + i * RPI * G::PITCH, ks + i * RPI * rowstride);
+        cp_async16(vdst + i * RPI * G::PITCH, vs + i * RPI * rowstride);
+      }
+      return;
+    }
+    // general tile: lane i resolves list position 32*tile + i to (tensor, element offset of its row)
+    const int p = tile * KT + lane;
+    int64_t off = -1;   // -1: no such position, the row is zero-filled
+    int which = 0;      // 0 shared segment, 1 private segment, 2 this step's k_new / v_new
+    if (lane >= KT) {
+      // no row for this lane in a tile of fewer than 32 positions
+    } else if (p < n_shared) {
+      off = (key_row(a.src, b, key_begin + p) * a.Hkv + kvh) * D;
+    } else if (p < n_total) {
+      const int pk = p - n_shared, w = w_lo + pk / step, t = pk % step;
+      const int64_t j = (int64_t)b * W + w;
+      if (t == step - 1) {
+        which = 2;
+        off = (j * a.Hkv + kvh) * D;
+      } else {
+        int64_t slab = j;
+        if (a.lineage) slab = min(max(a.lineage[j * a.max_new + t], 0), a.batch * W - 1);
+        which = 1;
+        off = ((slab * a.max_new + t) * a.Hkv + kvh) * D;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < NIT; ++i) {
+      const int64_t o_r = __shfl_sync(0xffffffffu, off, r0 + i * RPI);
+      const int w_r = __shfl_sync(0xffffffffu, which, r0 + i * RPI);
+      const bf16* ks = (w_r == 0 ? kg : w_r == 1 ? kp : kn) + (o_r < 0 ? 0 : o_r) + ch * 8;
+      const bf16* vs = (w_r == 0 ? vg : w_r == 1 ? vp : vn) + (o_r < 0 ? 0 : o_r) + ch * 8;
+      const int bytes = o_r < 0 ? 0 : 16;   // 0: nothing is read, the 16 destination bytes become zero
+      cp_async16(kdst + i * RPI * G::PITCH, ks, bytes);
+      cp_async16(vdst + i * RPI * G::PITCH, vs, bytes);
+    }
+  };
+
+  const int n_my = (n_tiles - warp + NWARPS - 1) / NWARPS;   // tiles warp, warp + NWARPS, ...
+#pragma unroll
+  for (int s = 0; s < STAGES - 1; ++s) {
+    if (s < n_my) issue_tile(warp + s * NWARPS, s);
+    cp_async_commit();
+  }
+
   // ---- Eq. 4: append.  Split 0 stores the new K/V row of every beam whose first query row is in this tile.
   if (split == 0) {
+    constexpr int CH = G::ROWB / 16;
     for (int w = w_lo; w <= w_hi; ++w) {
       if (w * g < row0) continue;   // that beam's first row belongs to the previous row tile
       const int64_t j = (int64_t)b * W + w;
@@ -102,64 +163,10 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
     }
   }
 
+  // ---- Q fragments (A operand, 16 rows x D), loaded while the first tiles are in flight; rows >= W*g are zero
   const int c2 = (lane & 3) * 2;
   const int rr0 = row0 + (lane >> 2), rr1 = rr0 + 8;
   const int beam0 = rr0 / g, beam1 = rr1 / g;
-
-  // ---- per-warp cp.async ring
-  uint8_t* ring = smem + warp * (STAGES * 2 * TILE_B);
-  const uint32_t ring_s = smem_addr(ring);
-
-  auto issue_tile = [&](int tile, int stage) {
-    const uint32_t kdst = ring_s + stage * 2 * TILE_B, vdst = kdst + TILE_B;
-#pragma unroll
-    for (int i = 0; i < KT * CH / 32; ++i) {
-      const int idx = lane + 32 * i, r = idx / CH, ch = idx % CH;
-      const bf16 *ks = kg, *vs = vg;
-      int bytes = 0;
-      if (tile < tiles_sh) {
-        const int key = key_begin + tile * KT + r;
-        if (key < key_end) {
-          const int64_t off = (key_row(a.src, b, key) * a.Hkv + kvh) * D + ch * 8;
-          ks = kg + off; vs = vg + off; bytes = 16;
-        }
-      } else {
-        const int pk = (tile - tiles_sh) * KT + r;
-        if (pk < n_priv) {
-          const int w = w_lo + pk / step, t = pk % step;
-          const int64_t j = (int64_t)b * W + w;
-          if (t == step - 1) {
-            const int64_t off = (j * a.Hkv + kvh) * D + ch * 8;
-            ks = kn + off; vs = vn + off;
-          } else {
-            int64_t slab = j;
-            if (a.lineage) slab = min(max(a.lineage[j * a.max_new + t], 0), a.batch * W - 1);
-            const int64_t off = ((slab * a.max_new + t) * a.Hkv + kvh) * D + ch * 8;
-            ks = kp + off; vs = vp + off;
-          }
-          bytes = 16;
-        }
-      }
-      const uint32_t so = r * ROWB + ((ch ^ (r & 7)) << 4);
-      cp_async16(kdst + so, ks, bytes);   // bytes == 0: the 16 destination bytes are zero-filled
-      cp_async16(vdst + so, vs, bytes);
-    }
-  };
-
-  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
-  float o[NTILES][4];
-#pragma unroll
-  for (int n = 0; n < NTILES; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
-
-  const int n_my = (n_tiles - warp + NWARPS - 1) / NWARPS;   // tiles warp, warp + NWARPS, ...
-#pragma unroll
-  for (int s = 0; s < STAGES - 1; ++s) {
-    if (s < n_my) issue_tile(warp + s * NWARPS, s);
-    cp_async_commit();
-  }
-
-  // ---- Q fragments (A operand, 16 rows x D), loaded while the first tiles are in flight;
-  //      rows beyond W*g are zero
   uint32_t qf[KSTEPS][4];
   {
     const bf16* qg = reinterpret_cast<const bf16*>(a.q);
@@ -177,76 +184,99 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
     }
   }
 
-  for (int it = 0; it < n_my; ++it) {
-    const int nxt = it + STAGES - 1;
-    if (nxt < n_my) issue_tile(warp + nxt * NWARPS, nxt % STAGES);
-    cp_async_commit();
-    cp_async_wait<STAGES - 1>();
-    __syncwarp();
-    const int tile = warp + it * NWARPS;
-    const uint32_t ks = ring_s + (it % STAGES) * 2 * TILE_B, vs = ks + TILE_B;
-
-    // S = Q K^T for 16 keys: two n-tiles of 8 keys
-    float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-    {
-      const int mat = lane >> 3, r = ((mat >> 1) << 3) + (lane & 7);
+  float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;   // running max in the scaled log2 domain
+  float o[NTILES][4];
 #pragma unroll
-      for (int kk = 0; kk < KSTEPS; ++kk) {
-        const int ch = kk * 2 + (mat & 1);
+  for (int n = 0; n < NTILES; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+
+  // ldmatrix lane addressing inside a tile (rows = keys, 16-byte chunks along d)
+  const int mat = lane >> 3;
+  const uint32_t k_lane = (uint32_t)(((mat >> 1) << 3) + (lane & 7)) * G::PITCH + (uint32_t)(mat & 1) * 16;
+  const uint32_t v_lane = (uint32_t)(((mat & 1) << 3) + (lane & 7)) * G::PITCH + (uint32_t)(mat >> 1) * 16;
+
+  for (int it = 0; it < n_my; ++it) {
+    const int stage = it % STAGES;
+    {
+      const int nxt = it + STAGES - 1;   // refill the stage that was consumed in the previous iteration
+      if (nxt < n_my) issue_tile(warp + nxt * NWARPS, nxt % STAGES);
+      cp_async_commit();
+      cp_async_wait<STAGES - 1>();       // this lane's copies of tile `it` have landed ...
+      __syncwarp();                      // ... and so have every other lane's
+    }
+    const int tile = warp + it * NWARPS;
+    const uint32_t ks = ring + stage * G::STAGE_B, vs = ks + G::TILE_B;
+
+    // S = Q K^T for KT positions: n-tiles of 8
+    float s[N8][4];
+#pragma unroll
+    for (int n = 0; n < N8; ++n) { s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f; }
+#pragma unroll
+    for (int kk = 0; kk < KSTEPS; ++kk) {
+#pragma unroll
+      for (int h16 = 0; h16 < H16; ++h16) {
         uint32_t b0, b1, b2, b3;
-        ldsm_x4(ks + r * ROWB + ((ch ^ (r & 7)) << 4), b0, b1, b2, b3);
-        mma_bf16(s[0], qf[kk], b0, b1);
-        mma_bf16(s[1], qf[kk], b2, b3);
+        ldsm_x4(ks + k_lane + h16 * 16 * G::PITCH + kk * 32, b0, b1, b2, b3);
+        mma_bf16(s[2 * h16], qf[kk], b0, b1);
+        mma_bf16(s[2 * h16 + 1], qf[kk], b2, b3);
       }
     }
-    // mask + scale
-    const bool priv = tile >= tiles_sh;
-    const int kbase = priv ? (tile - tiles_sh) * KT : key_begin + tile * KT;
+    // positions past the list, and generated tokens of other beams, are invisible
+    if ((tile + 1) * KT > n_shared) {
 #pragma unroll
-    for (int n = 0; n < 2; ++n)
+      for (int n = 0; n < N8; ++n)
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int key = kbase + n * 8 + c2 + (e & 1);
-        bool vis;
-        if (priv) vis = key < n_priv && (w_lo + key / step) == ((e < 2) ? beam0 : beam1);
-        else vis = key < key_end;
-        s[n][e] = vis ? s[n][e] * scale_log2 : -INFINITY;
-      }
-    float mx0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
-    float mx1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
+        for (int e = 0; e < 4; ++e) {
+          const int p = tile * KT + n * 8 + c2 + (e & 1);
+          bool vis = p < n_total;
+          if (p >= n_shared) vis = vis && (w_lo + (p - n_shared) / step) == ((e < 2) ? beam0 : beam1);
+          if (!vis) s[n][e] = -INFINITY;
+        }
+    }
+    float mx0 = fmaxf(s[0][0], s[0][1]), mx1 = fmaxf(s[0][2], s[0][3]);
+#pragma unroll
+    for (int n = 1; n < N8; ++n) {
+      mx0 = fmaxf(mx0, fmaxf(s[n][0], s[n][1]));
+      mx1 = fmaxf(mx1, fmaxf(s[n][2], s[n][3]));
+    }
     mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
     mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
     mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
     mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-    const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+    const float mn0 = fmaxf(m0, mx0 * scale_log2), mn1 = fmaxf(m1, mx1 * scale_log2);
     const float mu0 = (mn0 == -INFINITY) ? 0.f : mn0, mu1 = (mn1 == -INFINITY) ? 0.f : mn1;
-    const float al0 = exp2f(m0 - mu0), al1 = exp2f(m1 - mu1);
+    const float al0 = ex2(m0 - mu0), al1 = ex2(m1 - mu1);
+    const bool grew = (mn0 != m0) || (mn1 != m1);
     m0 = mn0; m1 = mn1;
-    uint32_t pf[4];
+    uint32_t pf[H16][4];
     {
-      const float p00 = exp2f(s[0][0] - mu0), p01 = exp2f(s[0][1] - mu0), p02 = exp2f(s[0][2] - mu1), p03 = exp2f(s[0][3] - mu1);
-      const float p10 = exp2f(s[1][0] - mu0), p11 = exp2f(s[1][1] - mu0), p12 = exp2f(s[1][2] - mu1), p13 = exp2f(s[1][3] - mu1);
-      l0 = l0 * al0 + (p00 + p01 + p10 + p11);   // per-lane partial sums; reduced over the quad at the end
-      l1 = l1 * al1 + (p02 + p03 + p12 + p13);
-      pf[0] = pack2(p00, p01); pf[1] = pack2(p02, p03); pf[2] = pack2(p10, p11); pf[3] = pack2(p12, p13);
+      float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+      for (int n = 0; n < N8; ++n) {
+        const float p0 = ex2(fmaf(s[n][0], scale_log2, -mu0)), p1 = ex2(fmaf(s[n][1], scale_log2, -mu0));
+        const float p2 = ex2(fmaf(s[n][2], scale_log2, -mu1)), p3 = ex2(fmaf(s[n][3], scale_log2, -mu1));
+        sum0 += p0 + p1; sum1 += p2 + p3;
+        pf[n >> 1][(n & 1) * 2] = pack2(p0, p1);
+        pf[n >> 1][(n & 1) * 2 + 1] = pack2(p2, p3);
+      }
+      l0 = l0 * al0 + sum0;   // per-lane partial sums; reduced over the quad at the end
+      l1 = l1 * al1 + sum1;
     }
-    // O = O * alpha + P V
-    {
-      const int mat = lane >> 3, r = ((mat & 1) << 3) + (lane & 7);
+    if (__any_sync(0xffffffffu, grew)) {
+#pragma unroll
+      for (int n = 0; n < NTILES; ++n) { o[n][0] *= al0; o[n][1] *= al0; o[n][2] *= al1; o[n][3] *= al1; }
+    }
+    // O += P V
+#pragma unroll
+    for (int h16 = 0; h16 < H16; ++h16) {
 #pragma unroll
       for (int nn = 0; nn < NTILES / 2; ++nn) {
-        const int ch = nn * 2 + (mat >> 1);
         uint32_t b0, b1, b2, b3;
-        ldsm_x4_t(vs + r * ROWB + ((ch ^ (r & 7)) << 4), b0, b1, b2, b3);
-        float* oa = o[2 * nn];
-        float* ob = o[2 * nn + 1];
-        oa[0] *= al0; oa[1] *= al0; oa[2] *= al1; oa[3] *= al1;
-        ob[0] *= al0; ob[1] *= al0; ob[2] *= al1; ob[3] *= al1;
-        mma_bf16(o[2 * nn], pf, b0, b1);
-        mma_bf16(o[2 * nn + 1], pf, b2, b3);
+        ldsm_x4_t(vs + v_lane + h16 * 16 * G::PITCH + nn * 32, b0, b1, b2, b3);
+        mma_bf16(o[2 * nn], pf[h16], b0, b1);
+        mma_bf16(o[2 * nn + 1], pf[h16], b2, b3);
       }
     }
-    __syncwarp();   // every lane is done with this stage before a later iteration refills it
+    __syncwarp();   // every lane is done with this stage before the next iteration refills it
   }
   cp_async_wait<0>();
   l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
@@ -313,61 +343,76 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
         if (threadIdx.x % GROUPS == 0) a.part_lse[prow] = big + log2f(den);
       }
     }
+    if (a.plan.n_splits <= 1) return;
+
+    // ---- the split that finishes last folds all partials of this (sequence, kv head, row tile).
+    // No CTA waits for another: each publishes its partial, takes a ticket, and only the holder of the
+    // last ticket reads the others' partials (which its ticket proves complete).
+    __threadfence();
+    __syncthreads();
+    int* is_last = reinterpret_cast<int*>(ml + NWARPS * 16 * 2);
+    int32_t* ticket = a.tickets + ((int64_t)(b * a.Hkv + kvh) * row_tiles + blockIdx.x % row_tiles);
+    const int live_splits = max(1, min(a.plan.n_splits, (shared_len + a.plan.chunk - 1) / a.plan.chunk));
+    if (threadIdx.x == 0) {
+      const int t = atomicAdd(ticket, 1);
+      *is_last = (t == live_splits - 1);
+      if (t == live_splits - 1) *ticket = 0;   // ready for the next launch on this stream
+    }
+    __syncthreads();
+    if (!*is_last) return;
+    __threadfence();
+    if (rr < n_rows) {
+      const int64_t prow0 = (int64_t)(b * a.Hkv + kvh) * a.plan.n_splits * a.plan.rows_pad + rr;
+      float top = -INFINITY;
+      for (int s = 0; s < live_splits; ++s) top = fmaxf(top, __ldcg(a.part_lse + prow0 + (int64_t)s * a.plan.rows_pad));
+      float den = 0.f, out[COLS];
+#pragma unroll
+      for (int c = 0; c < COLS; ++c) out[c] = 0.f;
+      for (int s = 0; s < live_splits; ++s) {
+        const int64_t prow = prow0 + (int64_t)s * a.plan.rows_pad;
+        const float wt = exp2f(__ldcg(a.part_lse + prow) - top);
+        den += wt;
+        const float4* po = reinterpret_cast<const float4*>(a.part_o + prow * D + cg);
+#pragma unroll
+        for (int c = 0; c < COLS; c += 4) {
+          const float4 x = __ldcg(po + c / 4);
+          out[c] += wt * x.x; out[c + 1] += wt * x.y; out[c + 2] += wt * x.z; out[c + 3] += wt * x.w;
+        }
+      }
+      const float inv = 1.f / den;
+      bf16* dst = reinterpret_cast<bf16*>(a.o) + (((int64_t)b * W + rr / g) * a.Hq + kvh * g + rr % g) * D + cg;
+#pragma unroll
+      for (int c = 0; c < COLS; c += 8) {
+        uint4 v;
+        v.x = pack2(out[c] * inv, out[c + 1] * inv); v.y = pack2(out[c + 2] * inv, out[c + 3] * inv);
+        v.z = pack2(out[c + 4] * inv, out[c + 5] * inv); v.w = pack2(out[c + 6] * inv, out[c + 7] * inv);
+        *reinterpret_cast<uint4*>(dst + c) = v;
+      }
+    }
   }
 }
 
-// Folds the split partials: one warp per (query row, kv head, sequence).
-template <int D>
-__global__ void __launch_bounds__(128) decode_combine_kernel(DecodeArgs a) {
-  constexpr int E = D / 32;
-  const int lane = threadIdx.x & 31;
-  const int rr = blockIdx.x * 4 + (threadIdx.x >> 5), kvh = blockIdx.y, b = blockIdx.z;
-  const int g = a.Hq / a.Hkv, W = a.beams;
-  if (rr >= W * g) return;
-  const int shared_len = a.src.paged ? a.src.n_regs : (a.cu_seqlens[b + 1] - a.cu_seqlens[b]);
-  const int64_t prow0 = (int64_t)(b * a.Hkv + kvh) * a.plan.n_splits * a.plan.rows_pad + rr;
-  float big = -INFINITY;
-  for (int s = 0; s < a.plan.n_splits; ++s)
-    if (s == 0 || s * a.plan.chunk < shared_len) big = fmaxf(big, a.part_lse[prow0 + (int64_t)s * a.plan.rows_pad]);
-  float den = 0.f, out[E];
-#pragma unroll
-  for (int e = 0; e < E; ++e) out[e] = 0.f;
-  for (int s = 0; s < a.plan.n_splits; ++s) {
-    if (!(s == 0 || s * a.plan.chunk < shared_len)) continue;
-    const int64_t prow = prow0 + (int64_t)s * a.plan.rows_pad;
-    const float wt = exp2f(a.part_lse[prow] - big);
-    den += wt;
-    const float* po = a.part_o + prow * D + lane * E;
-#pragma unroll
-    for (int e = 0; e < E; ++e) out[e] += wt * po[e];
-  }
-  __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.o) + (((int64_t)b * W + rr / g) * a.Hq + kvh * g + rr % g) * D + lane * E;
-  const float inv = 1.f / den;
-#pragma unroll
-  for (int e = 0; e < E; e += 2) *reinterpret_cast<uint32_t*>(dst + e) = pack2(out[e] * inv, out[e + 1] * inv);
-}
-
-template <int D>
+template <int D, int ST>
 cudaError_t launch_d(const DecodeArgs& a, cudaStream_t st) {
-  constexpr int smem = decode_smem_bytes<D>();
-  cudaError_t e = ensure_dynamic_smem<decode_mma_kernel<D>>(smem);
+  constexpr int smem = Geo<D, ST>::SMEM_B;
+  cudaError_t e = ensure_dynamic_smem<decode_mma_kernel<D, ST>>(smem);
   if (e != cudaSuccess) return e;
   const int splits = a.plan.n_splits > 0 ? a.plan.n_splits : 1;
   dim3 grid(splits * a.plan.row_tiles, a.Hkv, a.batch);
-  decode_mma_kernel<D><<<grid, NWARPS * 32, smem, st>>>(a);
-  note_launch();
-  e = cudaGetLastError();
-  if (e != cudaSuccess || a.plan.n_splits <= 1) return e;
-  dim3 cgrid((a.plan.rows + 3) / 4, a.Hkv, a.batch);
-  decode_combine_kernel<D><<<cgrid, 128, 0, st>>>(a);
+  decode_mma_kernel<D, ST><<<grid, NWARPS * 32, smem, st>>>(a);
   note_launch();
   return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
-  return a.D == 64 ? launch_d<64>(a, st) : launch_d<128>(a, st);
+cudaError_t launch_decode_mma(const DecodeArgs& a, int max_shared_len, cudaStream_t st) {
+  // a key list of at most two tiles needs no deep ring: a small footprint keeps every CTA resident at once
+  const int g = a.Hq / a.Hkv;
+  const int beams_per_tile = a.beams < (16 + g - 1) / g + 1 ? a.beams : (16 + g - 1) / g + 1;
+  const bool small = a.plan.n_splits <= 1 && max_shared_len + beams_per_tile * a.step <= 2 * KT * NWARPS;
+  if (a.D == 64) return small ? launch_d<64, 2>(a, st) : launch_d<64, EARN_DECODE_STAGES>(a, st);
+  return small ? launch_d<128, 2>(a, st) : launch_d<128, EARN_DECODE_STAGES>(a, st);
 }
 
 }  // namespace earn

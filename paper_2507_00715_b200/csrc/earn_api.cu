@@ -56,10 +56,11 @@ DecodePlan make_decode_plan(const earn_model_t& m, const earn_batch_t& b, int be
   p.row_tiles = (p.rows + kDecodeRows - 1) / kDecodeRows;
   p.rows_pad = p.row_tiles * kDecodeRows;
   if (max_shared_len <= 0 || b.batch == 0) { p.chunk = 64; p.n_splits = 0; return p; }
-  // enough CTAs to cover the SMs a few times over, but no more splits than that needs
+  // Split only while the unsplit CTAs would leave resident slots empty (six decode CTAs fit an SM): on B200
+  // every extra split of the 7B shapes cost time (50.9 us unsplit, 65.8 us in two splits).
   const long units = (long)b.batch * m.n_kv_heads * p.row_tiles;
-  const long want = 3L * 148;   // four decode CTAs fit an SM; aim for most of those slots in one wave
-  long splits = (want + units - 1) / units;
+  const long slots = 6L * 148;
+  long splits = slots / units;
   long max_splits = (max_shared_len + 63) / 64;
   if (splits > max_splits) splits = max_splits;
   if (splits < 1) splits = 1;
@@ -72,11 +73,16 @@ size_t decode_partial_floats(const earn_model_t& m, const earn_batch_t& b, const
   return (size_t)b.batch * m.n_kv_heads * p.n_splits * p.rows_pad * (size_t)(m.head_dim + 1);
 }
 
+// one int32 ticket per (sequence, kv head, row tile), after the status word
+static size_t ticket_bytes(const earn_model_t& m, const earn_batch_t& b, const DecodePlan& p) {
+  return round_up(sizeof(int32_t) * (size_t)b.batch * m.n_kv_heads * p.row_tiles, 256);
+}
+
 static size_t workspace_need(const earn_model_t* m, const earn_batch_t* b, int beams) {
   DecodePlan full = make_decode_plan(*m, *b, beams, b->max_seqlen);
   DecodePlan reg = make_decode_plan(*m, *b, beams, b->n_head_reg + b->n_tail_reg);
   size_t f = decode_partial_floats(*m, *b, full), r = decode_partial_floats(*m, *b, reg);
-  return kStatusBytes + round_up(sizeof(float) * (f > r ? f : r), 256) + 256;
+  return kStatusBytes + ticket_bytes(*m, *b, full) + round_up(sizeof(float) * (f > r ? f : r), 256) + 256;
 }
 
 static earn_status_t check_cache_shared(const earn_model_t* m, const earn_batch_t* b, const earn_cache_t* c) {
@@ -130,7 +136,8 @@ size_t earn_workspace_bytes(const earn_model_t* model, const earn_batch_t* batch
 
 earn_status_t earn_workspace_init(void* workspace, size_t workspace_bytes, earn_stream_t stream) {
   if (workspace == nullptr || workspace_bytes < (size_t)kStatusBytes || !aligned16(workspace)) return EARN_ERR_WORKSPACE;
-  return cudaMemsetAsync(workspace, 0, kStatusBytes, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+  // status word and split tickets start at zero (the partial buffers behind them need no value)
+  return cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
 }
 
 earn_status_t earn_device_status(const void* workspace, earn_stream_t stream) {
@@ -255,12 +262,13 @@ earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* ba
   a.k_priv = cache->k_priv; a.v_priv = cache->v_priv; a.lineage = cache->lineage;
   a.plan = make_decode_plan(*model, *batch, cache->beams,
                             early ? batch->max_seqlen : batch->n_head_reg + batch->n_tail_reg);
-  a.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) + kStatusBytes);
+  a.tickets = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(workspace) + kStatusBytes);
+  a.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) + kStatusBytes + ticket_bytes(*model, *batch, a.plan));
   a.part_lse = a.part_o + (size_t)batch->batch * model->n_kv_heads * a.plan.n_splits * a.plan.rows_pad * model->head_dim;
   a.batch = batch->batch; a.beams = cache->beams; a.max_new = cache->max_new; a.step = step;
   a.Hq = model->n_q_heads; a.Hkv = model->n_kv_heads; a.D = model->head_dim; a.dtype = model->dtype;
   a.scale = scale_of(model);
-  const cudaError_t e = model->dtype == EARN_BF16 ? launch_decode_mma(a, (cudaStream_t)stream)
+  const cudaError_t e = model->dtype == EARN_BF16 ? launch_decode_mma(a, early ? batch->max_seqlen : batch->n_head_reg + batch->n_tail_reg, (cudaStream_t)stream)
                                                    : launch_decode_simt(a, (cudaStream_t)stream);
   return e == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
 }

@@ -95,12 +95,14 @@ struct DecodeArgs {
   const int32_t* lineage;
   float* part_o;               // [B, Hkv, n_splits, rows_pad, D]
   float* part_lse;             // [B, Hkv, n_splits, rows_pad]  (log2 domain)
+  int32_t* tickets;            // [B, Hkv, row_tiles], zero between launches: which split finished last
   DecodePlan plan;
   int batch, beams, max_new, step, Hq, Hkv, D, dtype;
   float scale;
 };
 cudaError_t launch_decode_simt(const DecodeArgs& a, cudaStream_t st);   // fp32 debug path
-cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st);    // bf16: cp.async rings + mma.sync
+// bf16: cp.async ring + mma.sync; max_shared_len = longest shared segment of the batch (picks the ring depth)
+cudaError_t launch_decode_mma(const DecodeArgs& a, int max_shared_len, cudaStream_t st);
 
 struct CompactArgs {
   const void *k, *v, *q;
