@@ -221,7 +221,9 @@ earn_status_t earn_register_attn(const earn_model_t* model, const earn_batch_t* 
   a.batch = batch->batch; a.R = R;
   a.Hq = model->n_q_heads; a.Hkv = model->n_kv_heads; a.D = model->head_dim; a.dtype = model->dtype;
   a.scale = scale_of(model);
-  return launch_register_simt(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+  const cudaError_t e = register_mma_supported(a) ? launch_register_mma(a, (cudaStream_t)stream)
+                                                  : launch_register_simt(a, (cudaStream_t)stream);
+  return e == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
 }
 
 earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, int32_t step,

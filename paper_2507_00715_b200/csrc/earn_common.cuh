@@ -85,6 +85,8 @@ struct RegisterArgs {
   float scale;
 };
 cudaError_t launch_register_simt(const RegisterArgs& a, cudaStream_t st);
+bool register_mma_supported(const RegisterArgs& a);                      // bf16 and R <= 128
+cudaError_t launch_register_mma(const RegisterArgs& a, cudaStream_t st);
 
 struct DecodeArgs {
   const void *q, *k_new, *v_new;

@@ -1,0 +1,186 @@
+// Register-only attention of a layer l >= k during prefill (Section 3.2, register-focused process):
+// causal attention among the R compact register rows of each sequence, order [prefix; suffix].
+//
+// The work per sequence is tiny (R <= 128 keys), so the kernel is shaped for HBM traffic and latency:
+// one CTA per (sequence, kv head) brings that head's compact K and V rows into shared memory once
+// (through the page table) and all g query heads of the group use them.  The g*R query rows
+// (row = head-in-group * R + register index) are cut into tiles of 16; each of the 8 warps takes
+// tiles round-robin, keeps its Q fragments in registers, runs mma.sync m16n8k16 over 16-key tiles up
+// to the causal limit with an online softmax in the log2 domain, and writes its 16 output rows
+// through a private shared-memory staging tile as 16-byte stores.
+#include "earn_common.cuh"
+#include "mma_sync.cuh"
+#include "sm100_ptx.cuh"
+
+namespace earn {
+namespace {
+using namespace mma;
+
+constexpr int NW = 8;
+constexpr int MAX_R = 128;
+
+template <int D>
+struct RGeo {
+  static constexpr int ROWB = D * 2;
+  static constexpr int PITCH = ROWB + 16;
+};
+
+template <int D>
+__global__ void __launch_bounds__(NW * 32) register_mma_kernel(RegisterArgs a, int r_pad) {
+  using bf16 = __nv_bfloat16;
+  using G = RGeo<D>;
+  constexpr int KSTEPS = D / 16, NTILES = D / 8, CH = G::ROWB / 16;
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kvh = blockIdx.x, b = blockIdx.y;
+  const int R = a.R, g = a.Hq / a.Hkv, n_rows = g * R;
+  const uint32_t sK = ptx::smem_u32(smem), sV = sK + r_pad * G::PITCH;
+  uint8_t* gO = smem + 2 * r_pad * G::PITCH + warp * 16 * G::PITCH;
+
+  // ---- compact K/V rows of this (sequence, kv head) -> shared memory; rows R..r_pad-1 are zero
+  {
+    const bf16* kg = reinterpret_cast<const bf16*>(a.src.k);
+    const bf16* vg = reinterpret_cast<const bf16*>(a.src.v);
+    for (int i = threadIdx.x; i < r_pad * CH; i += NW * 32) {
+      const int r = i / CH, ch = i % CH;
+      const int64_t off = r < R ? (key_row(a.src, b, r) * a.Hkv + kvh) * D + ch * 8 : 0;
+      const int bytes = r < R ? 16 : 0;
+      cp_async16(sK + r * G::PITCH + ch * 16, kg + off, bytes);
+      cp_async16(sV + r * G::PITCH + ch * 16, vg + off, bytes);
+    }
+    cp_async_commit();
+  }
+
+  const float scale_log2 = a.scale * kLog2e;
+  const int c2 = (lane & 3) * 2;
+  const int mat = lane >> 3;
+  const uint32_t k_lane = (uint32_t)(((mat >> 1) << 3) + (lane & 7)) * G::PITCH + (uint32_t)(mat & 1) * 16;
+  const uint32_t v_lane = (uint32_t)(((mat & 1) << 3) + (lane & 7)) * G::PITCH + (uint32_t)(mat >> 1) * 16;
+  const bf16* qg = reinterpret_cast<const bf16*>(a.q_reg);
+  bf16* og = reinterpret_cast<bf16*>(a.o_reg);
+  cp_async_wait<0>();
+  __syncthreads();   // every warp's copies have landed (warps without a tile take part too)
+
+  for (int tile = warp; tile * 16 < n_rows; tile += NW) {
+    const int rr0 = tile * 16 + (lane >> 2), rr1 = rr0 + 8;
+    // row -> (head in group, register index); rows past g*R read nothing and write nothing
+    const int gi0 = rr0 / R, m0r = rr0 % R, gi1 = rr1 / R, m1r = rr1 % R;
+    const bool ok0 = rr0 < n_rows, ok1 = rr1 < n_rows;
+    uint32_t qf[KSTEPS][4];
+    {
+      const bf16* q0 = qg + (((int64_t)b * R + m0r) * a.Hq + kvh * g + gi0) * D;
+      const bf16* q1 = qg + (((int64_t)b * R + m1r) * a.Hq + kvh * g + gi1) * D;
+#pragma unroll
+      for (int kk = 0; kk < KSTEPS; ++kk) {
+        qf[kk][0] = ok0 ? *reinterpret_cast<const uint32_t*>(q0 + kk * 16 + c2) : 0u;
+        qf[kk][1] = ok1 ? *reinterpret_cast<const uint32_t*>(q1 + kk * 16 + c2) : 0u;
+        qf[kk][2] = ok0 ? *reinterpret_cast<const uint32_t*>(q0 + kk * 16 + 8 + c2) : 0u;
+        qf[kk][3] = ok1 ? *reinterpret_cast<const uint32_t*>(q1 + kk * 16 + 8 + c2) : 0u;
+      }
+    }
+    // causal limit of the tile: the largest register index among its rows
+    const int first = tile * 16, last = min(first + 15, n_rows - 1);
+    const int m_hi = (first / R == last / R) ? last % R : R - 1;
+    const int key_tiles = m_hi / 16 + 1;
+
+    float mx0 = -INFINITY, mx1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    float o[NTILES][4];
+#pragma unroll
+    for (int n = 0; n < NTILES; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
+
+    for (int kt = 0; kt < key_tiles; ++kt) {
+      const uint32_t ks = sK + kt * 16 * G::PITCH, vs = sV + kt * 16 * G::PITCH;
+      float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+      for (int kk = 0; kk < KSTEPS; ++kk) {
+        uint32_t b0, b1, b2, b3;
+        ldsm_x4(ks + k_lane + kk * 32, b0, b1, b2, b3);
+        mma_bf16(s[0], qf[kk], b0, b1);
+        mma_bf16(s[1], qf[kk], b2, b3);
+      }
+#pragma unroll
+      for (int n = 0; n < 2; ++n)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int j = kt * 16 + n * 8 + c2 + (e & 1);
+          if (j > ((e < 2) ? m0r : m1r)) s[n][e] = -INFINITY;   // key after the row's own register (also j >= R)
+        }
+      float t0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
+      float t1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
+      t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, 1));
+      t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, 2));
+      t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, 1));
+      t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, 2));
+      const float mn0 = fmaxf(mx0, t0 * scale_log2), mn1 = fmaxf(mx1, t1 * scale_log2);
+      const float mu0 = (mn0 == -INFINITY) ? 0.f : mn0, mu1 = (mn1 == -INFINITY) ? 0.f : mn1;
+      const float al0 = ex2(mx0 - mu0), al1 = ex2(mx1 - mu1);
+      mx0 = mn0; mx1 = mn1;
+      uint32_t pf[4];
+      {
+        const float p00 = ex2(fmaf(s[0][0], scale_log2, -mu0)), p01 = ex2(fmaf(s[0][1], scale_log2, -mu0));
+        const float p02 = ex2(fmaf(s[0][2], scale_log2, -mu1)), p03 = ex2(fmaf(s[0][3], scale_log2, -mu1));
+        const float p10 = ex2(fmaf(s[1][0], scale_log2, -mu0)), p11 = ex2(fmaf(s[1][1], scale_log2, -mu0));
+        const float p12 = ex2(fmaf(s[1][2], scale_log2, -mu1)), p13 = ex2(fmaf(s[1][3], scale_log2, -mu1));
+        l0 = l0 * al0 + (p00 + p01 + p10 + p11);
+        l1 = l1 * al1 + (p02 + p03 + p12 + p13);
+        pf[0] = pack2(p00, p01); pf[1] = pack2(p02, p03); pf[2] = pack2(p10, p11); pf[3] = pack2(p12, p13);
+      }
+#pragma unroll
+      for (int nn = 0; nn < NTILES / 2; ++nn) {
+        uint32_t b0, b1, b2, b3;
+        ldsm_x4_t(vs + v_lane + nn * 32, b0, b1, b2, b3);
+        float* oa = o[2 * nn];
+        float* ob = o[2 * nn + 1];
+        oa[0] *= al0; oa[1] *= al0; oa[2] *= al1; oa[3] *= al1;
+        ob[0] *= al0; ob[1] *= al0; ob[2] *= al1; ob[3] *= al1;
+        mma_bf16(o[2 * nn], pf, b0, b1);
+        mma_bf16(o[2 * nn + 1], pf, b2, b3);
+      }
+    }
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    const float i0 = 1.f / l0, i1 = 1.f / l1;   // every row sees at least its own key
+    // ---- stage the 16 x D bf16 tile, then 16-byte stores (a row = D*2 contiguous bytes of o_reg)
+    __syncwarp();
+    {
+      const int r0 = lane >> 2, r1 = r0 + 8;
+#pragma unroll
+      for (int n = 0; n < NTILES; ++n) {
+        *reinterpret_cast<uint32_t*>(gO + r0 * G::PITCH + (n * 8 + c2) * 2) = pack2(o[n][0] * i0, o[n][1] * i0);
+        *reinterpret_cast<uint32_t*>(gO + r1 * G::PITCH + (n * 8 + c2) * 2) = pack2(o[n][2] * i1, o[n][3] * i1);
+      }
+    }
+    __syncwarp();
+    for (int i = lane; i < 16 * CH; i += 32) {
+      const int r = i / CH, ch = i % CH, rr = tile * 16 + r;
+      if (rr < n_rows) {
+        const uint4 v = *reinterpret_cast<const uint4*>(gO + r * G::PITCH + ch * 16);
+        *reinterpret_cast<uint4*>(og + (((int64_t)b * R + rr % R) * a.Hq + kvh * g + rr / R) * D + ch * 8) = v;
+      }
+    }
+  }
+}
+
+template <int D>
+cudaError_t launch_r(const RegisterArgs& a, cudaStream_t st) {
+  const int r_pad = (a.R + 15) / 16 * 16;
+  const int smem = 2 * r_pad * RGeo<D>::PITCH + NW * 16 * RGeo<D>::PITCH;
+  cudaError_t e = ensure_dynamic_smem<register_mma_kernel<D>>(2 * MAX_R * RGeo<D>::PITCH + NW * 16 * RGeo<D>::PITCH);
+  if (e != cudaSuccess) return e;
+  dim3 grid(a.Hkv, a.batch);
+  register_mma_kernel<D><<<grid, NW * 32, smem, st>>>(a, r_pad);
+  note_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool register_mma_supported(const RegisterArgs& a) { return a.dtype == EARN_BF16 && a.R <= MAX_R; }
+
+cudaError_t launch_register_mma(const RegisterArgs& a, cudaStream_t st) {
+  return a.D == 64 ? launch_r<64>(a, st) : launch_r<128>(a, st);
+}
+
+}  // namespace earn

@@ -52,3 +52,11 @@ def test_split_at_the_ends(k):
 
 def test_mha_and_many_registers():
     run_workload_and_compare(BASE.replace(seed=19, n_q_heads=2, n_kv_heads=2, r_head=40, r_tail=37, lens=(100, 300), batch=2))
+    # more than 128 registers: the register layers fall back to the CUDA-core kernel
+    run_workload_and_compare(BASE.replace(seed=20, n_q_heads=4, n_kv_heads=2, r_head=70, r_tail=75, lens=(150, 300), batch=2))
+
+
+def test_group_of_three_and_odd_register_count():
+    # g*R = 3*7 = 21 rows: a ragged last row tile that straddles two heads
+    run_workload_and_compare(BASE.replace(seed=21, n_q_heads=6, n_kv_heads=2, r_head=3, r_tail=4, lens=(60, 33), batch=2,
+                                          beams=2, decode_steps=4))
