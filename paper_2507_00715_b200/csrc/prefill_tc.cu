@@ -1,15 +1,17 @@
 // Full causal prefill attention (Eq. 3 + causal mask, layers l < k) on the Blackwell tensor cores.
 // bf16 Q/K/V, head_dim 128, fp32 logits / softmax / accumulation, bf16 output.
 //
-// One CTA = 128 query rows of one (sequence, query head).  Per 128-key tile:
-//   TMA      : K and V tiles -> shared memory (128-byte swizzle), two stages
-//   tcgen05  : S = Q K^T into tensor memory (TMEM columns 0..127), issued by one thread
-//   softmax  : 128 threads, one query row each: read S from TMEM, online softmax in the log2 domain,
-//              write P as bf16 into swizzled shared memory
-//   tcgen05  : O += P V into TMEM columns 128..255
-// The running output stays in TMEM.  The softmax reference maximum is only raised when the row maximum
-// grows by more than 2^8; then the owning warp rescales its 32 rows of O in TMEM.  Exact after the
-// final division by the row sum.
+// One CTA = 128 query rows of NT query heads that share a kv head (NT = 2 when the GQA group size is
+// even, else 1): NT "M-tiles" with the same rows and the same key range, so they share every K/V tile
+// and finish together.  Per 128-key tile:
+//   warp 0     TMA: K and V tiles -> shared memory (128-byte swizzle), a ring of 32 KB entries K0 V0 K1 V1 ..
+//   warp 1     one thread issues tcgen05.mma: S_x = Q_x K^T into tensor memory, later O_x += P_x V
+//   warps 4..  one softmax warpgroup per M-tile, one query row per thread: read S_x from TMEM, online softmax
+//              in the log2 domain, write P_x as bf16 into swizzled shared memory
+// With two M-tiles the tensor core works on one while the other is in its softmax (S_A, S_B, O_A, O_B fill
+// the 512 TMEM columns).  The running output stays in TMEM.  The softmax reference maximum is only raised
+// when the row maximum grows by more than 2^8; then the owning warp rescales its 32 rows of O in TMEM.
+// Exact after the final division by the row sum.
 //
 // Every mbarrier wait is bounded; when one runs out the CTA raises its abort flag, writes
 // EARN_ERR_TIMEOUT to the status word, drains what it has in flight, frees its TMEM and returns.
@@ -25,18 +27,23 @@ using namespace ptx;
 constexpr int BM = 128, BN = 128, HD = 128;
 constexpr int TILE = BM * HD * 2;   // bytes of one 128 x 128 bf16 tile
 constexpr int HALF = TILE / 2;      // one 64-column block of it (128 rows x 128 B)
-constexpr int KV_STAGES = 2;
-constexpr int OFF_Q = 0;
-constexpr int OFF_K = OFF_Q + TILE;
-constexpr int OFF_V = OFF_K + KV_STAGES * TILE;
-constexpr int OFF_P = OFF_V + KV_STAGES * TILE;
-constexpr int OFF_BAR = OFF_P + TILE;
-constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;   // + alignment slack
-constexpr int TMEM_COLS = 256;
 constexpr long long WAIT_LIMIT = 2000000000LL;     // about one second of SM clocks
 constexpr float RESCALE_THRESHOLD = 8.f;           // log2 units
 
-enum { BAR_Q = 0, BAR_K = 1, BAR_V = 3, BAR_KV_EMPTY = 5, BAR_S = 7, BAR_P = 8, BAR_O = 9, BAR_DRAIN = 10, N_BARS = 11 };
+template <int NT>
+struct Cfg {
+  static constexpr int NSTAGE = NT == 1 ? 4 : 3;            // ring entries (K and V tiles alternate)
+  static constexpr int OFF_Q = 0;
+  static constexpr int OFF_RING = OFF_Q + NT * TILE;
+  static constexpr int OFF_P = OFF_RING + NSTAGE * TILE;
+  static constexpr int OFF_BAR = OFF_P + NT * TILE;
+  static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;   // + alignment slack
+  static constexpr int TMEM_COLS = NT * 256;                // S_x at x*128, O_x at (NT + x)*128
+  static constexpr int THREADS = 32 * (4 + 4 * NT);
+  // barriers
+  static constexpr int BAR_Q = 0, BAR_FULL = 1, BAR_EMPTY = BAR_FULL + NSTAGE, BAR_S = BAR_EMPTY + NSTAGE,
+                       BAR_P = BAR_S + NT, BAR_O = BAR_P + NT, BAR_DRAIN = BAR_O + NT, N_BARS = BAR_DRAIN + 1;
+};
 
 struct TcParams {
   void* o;
@@ -47,37 +54,40 @@ struct TcParams {
   float scale_log2;
 };
 
-__global__ void __launch_bounds__(192, 1)
+template <int NT>
+__global__ void __launch_bounds__(Cfg<NT>::THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, TcParams p) {
-  const int b = blockIdx.z, h = blockIdx.y;
+  using C = Cfg<NT>;
+  const int b = blockIdx.z, h0 = blockIdx.y * NT;
   const int lo = p.cu_seqlens[b], L = p.cu_seqlens[b + 1] - lo;
   const int q0 = ((int)gridDim.x - 1 - (int)blockIdx.x) * BM;   // longest tiles first
   if (q0 >= L) return;
   const int n_tiles = q0 / BN + 1;                                // causal: key tiles 0 .. diagonal
-  const int kvh = h / p.g;
+  const int kvh = h0 / p.g;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;    // swizzled tiles need 1024-byte alignment
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t sQ = base + OFF_Q, sK = base + OFF_K, sV = base + OFF_V, sP = base + OFF_P;
-  const uint32_t bars = base + OFF_BAR;
+  const uint32_t sQ = base + C::OFF_Q, sRing = base + C::OFF_RING, sP = base + C::OFF_P;
+  const uint32_t bars = base + C::OFF_BAR;
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + OFF_BAR + 8 * N_BARS);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + OFF_BAR + 8 * N_BARS + 8);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + C::OFF_BAR + 8 * C::N_BARS);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + C::OFF_BAR + 8 * C::N_BARS + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    mbar_init(bar(BAR_Q), 1);
-    for (int s = 0; s < KV_STAGES; ++s) {
-      mbar_init(bar(BAR_K + s), 1);
-      mbar_init(bar(BAR_V + s), 1);
-      mbar_init(bar(BAR_KV_EMPTY + s), 1);
+    mbar_init(bar(C::BAR_Q), 1);
+    for (int s = 0; s < C::NSTAGE; ++s) {
+      mbar_init(bar(C::BAR_FULL + s), 1);
+      mbar_init(bar(C::BAR_EMPTY + s), 1);
     }
-    mbar_init(bar(BAR_S), 1);
-    mbar_init(bar(BAR_P), 128);
-    mbar_init(bar(BAR_O), 1);
-    mbar_init(bar(BAR_DRAIN), 1);
+    for (int x = 0; x < NT; ++x) {
+      mbar_init(bar(C::BAR_S + x), 1);
+      mbar_init(bar(C::BAR_P + x), 128);
+      mbar_init(bar(C::BAR_O + x), 1);
+    }
+    mbar_init(bar(C::BAR_DRAIN), 1);
     *abort_flag = 0;
     fence_barrier_init();
     tma_prefetch_desc(&map_q);
@@ -85,42 +95,41 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     tma_prefetch_desc(&map_v);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), TMEM_COLS);
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), C::TMEM_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  const int n_entries = 2 * n_tiles;   // ring entries: K_0 V_0 K_1 V_1 ...
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      mbar_expect_tx(bar(BAR_Q), TILE);
-      tma_load_3d(sQ, &map_q, bar(BAR_Q), 0, h, lo + q0);
-      tma_load_3d(sQ + HALF, &map_q, bar(BAR_Q), 64, h, lo + q0);
+      mbar_expect_tx(bar(C::BAR_Q), NT * TILE);
+      for (int x = 0; x < NT; ++x) {
+        tma_load_3d(sQ + x * TILE, &map_q, bar(C::BAR_Q), 0, h0 + x, lo + q0);
+        tma_load_3d(sQ + x * TILE + HALF, &map_q, bar(C::BAR_Q), 64, h0 + x, lo + q0);
+      }
       int issued = 0;
-      bool ok = true;
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int st = j % KV_STAGES;
-        if (j >= KV_STAGES) ok = mbar_wait_bounded(bar(BAR_KV_EMPTY + st), ((j / KV_STAGES) - 1) & 1, abort_flag, WAIT_LIMIT);
-        if (!ok) break;
-        mbar_expect_tx(bar(BAR_K + st), TILE);
-        tma_load_3d(sK + st * TILE, &map_k, bar(BAR_K + st), 0, kvh, lo + j * BN);
-        tma_load_3d(sK + st * TILE + HALF, &map_k, bar(BAR_K + st), 64, kvh, lo + j * BN);
-        mbar_expect_tx(bar(BAR_V + st), TILE);
-        tma_load_3d(sV + st * TILE, &map_v, bar(BAR_V + st), 0, kvh, lo + j * BN);
-        tma_load_3d(sV + st * TILE + HALF, &map_v, bar(BAR_V + st), 64, kvh, lo + j * BN);
-        issued = j + 1;
+      for (int e = 0; e < n_entries; ++e) {
+        const int st = e % C::NSTAGE;
+        if (e >= C::NSTAGE &&
+            !mbar_wait_bounded(bar(C::BAR_EMPTY + st), ((e / C::NSTAGE) - 1) & 1, abort_flag, WAIT_LIMIT))
+          break;
+        const CUtensorMap* map = (e & 1) ? &map_v : &map_k;
+        mbar_expect_tx(bar(C::BAR_FULL + st), TILE);
+        tma_load_3d(sRing + st * TILE, map, bar(C::BAR_FULL + st), 0, kvh, lo + (e >> 1) * BN);
+        tma_load_3d(sRing + st * TILE + HALF, map, bar(C::BAR_FULL + st), 64, kvh, lo + (e >> 1) * BN);
+        issued = e + 1;
       }
       if (*abort_flag) {
         // let the copies already in flight land before the CTA gives its shared memory back
         int none = 0;
-        mbar_wait_bounded(bar(BAR_Q), 0, &none, WAIT_LIMIT);
-        for (int j = max(issued - KV_STAGES, 0); j < issued; ++j) {
-          mbar_wait_bounded(bar(BAR_K + j % KV_STAGES), (j / KV_STAGES) & 1, &none, WAIT_LIMIT);
-          mbar_wait_bounded(bar(BAR_V + j % KV_STAGES), (j / KV_STAGES) & 1, &none, WAIT_LIMIT);
-        }
+        mbar_wait_bounded(bar(C::BAR_Q), 0, &none, WAIT_LIMIT);
+        for (int e = max(issued - C::NSTAGE, 0); e < issued; ++e)
+          mbar_wait_bounded(bar(C::BAR_FULL + e % C::NSTAGE), (e / C::NSTAGE) & 1, &none, WAIT_LIMIT);
       }
     }
   } else if (warp == 1) {
@@ -128,53 +137,77 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     if (lane == 0) {
       constexpr uint32_t idesc_s = idesc_bf16_f32(BM, BN, 0, 0);   // Q (K-major) x K^T (K-major)
       constexpr uint32_t idesc_o = idesc_bf16_f32(BM, HD, 0, 1);   // P (K-major) x V (MN-major)
-      bool ok = mbar_wait_bounded(bar(BAR_Q), 0, abort_flag, WAIT_LIMIT);
-      for (int j = 0; j < n_tiles && ok; ++j) {
-        const int st = j % KV_STAGES, ph = (j / KV_STAGES) & 1;
-        ok = mbar_wait_bounded(bar(BAR_K + st), ph, abort_flag, WAIT_LIMIT);
-        if (!ok) break;
-        tc_fence_after();
+      auto wait_full = [&](int e) {
+        return mbar_wait_bounded(bar(C::BAR_FULL + e % C::NSTAGE), (e / C::NSTAGE) & 1, abort_flag, WAIT_LIMIT);
+      };
+      auto issue_s = [&](int x, int e) {   // S_x = Q_x K^T with the K tile of ring entry e
+        const uint32_t sK = sRing + (e % C::NSTAGE) * TILE;
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk) {
           const uint32_t off = (kk >> 2) * HALF + (kk & 3) * 32;
-          umma_ss(tmem, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + st * TILE + off, 16, 1024), idesc_s, kk > 0);
+          umma_ss(tmem + x * 128, smem_desc_sw128(sQ + x * TILE + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024),
+                  idesc_s, kk > 0);
         }
-        umma_commit(bar(BAR_S));
-        ok = mbar_wait_bounded(bar(BAR_P), j & 1, abort_flag, WAIT_LIMIT) &&
-             mbar_wait_bounded(bar(BAR_V + st), ph, abort_flag, WAIT_LIMIT);
-        if (!ok) break;
-        tc_fence_after();
+        umma_commit(bar(C::BAR_S + x));
+        if (x == NT - 1) umma_commit(bar(C::BAR_EMPTY + e % C::NSTAGE));   // K tile free once the last S has read it
+      };
+      auto issue_pv = [&](int x, int e, bool first) {   // O_x (+)= P_x V with the V tile of ring entry e
+        const uint32_t sV = sRing + (e % C::NSTAGE) * TILE;
 #pragma unroll
         for (int kk = 0; kk < BN / 16; ++kk) {
           const uint32_t offp = (kk >> 2) * HALF + (kk & 3) * 32;
-          umma_ss(tmem + 128, smem_desc_sw128(sP + offp, 16, 1024), smem_desc_sw128(sV + st * TILE + kk * 2048, HALF, 1024),
-                  idesc_o, (j > 0 || kk > 0) ? 1u : 0u);
+          umma_ss(tmem + (NT + x) * 128, smem_desc_sw128(sP + x * TILE + offp, 16, 1024),
+                  smem_desc_sw128(sV + kk * 2048, HALF, 1024), idesc_o, (!first || kk > 0) ? 1u : 0u);
         }
-        umma_commit(bar(BAR_KV_EMPTY + st));
-        if (j == n_tiles - 1) umma_commit(bar(BAR_O));
+        if (x == NT - 1) umma_commit(bar(C::BAR_EMPTY + e % C::NSTAGE));   // V tile free once the last P V has read it
+      };
+      bool ok = mbar_wait_bounded(bar(C::BAR_Q), 0, abort_flag, WAIT_LIMIT) && wait_full(0);
+      if (ok) {
+        tc_fence_after();
+        for (int x = 0; x < NT; ++x) issue_s(x, 0);
+      }
+      for (int j = 0; j < n_tiles && ok; ++j) {
+        for (int x = 0; x < NT && ok; ++x) {
+          ok = mbar_wait_bounded(bar(C::BAR_P + x), j & 1, abort_flag, WAIT_LIMIT);   // P_x(j) written, S_x free
+          if (ok && x == 0) ok = wait_full(2 * j + 1);
+          if (!ok) break;
+          tc_fence_after();
+          issue_pv(x, 2 * j + 1, j == 0);
+          if (j == n_tiles - 1) {
+            umma_commit(bar(C::BAR_O + x));
+          } else {
+            if (x == 0) ok = wait_full(2 * j + 2);
+            if (!ok) break;
+            tc_fence_after();
+            issue_s(x, 2 * j + 2);
+          }
+        }
       }
       if (*abort_flag) {
         int none = 0;
-        umma_commit(bar(BAR_DRAIN));   // everything this thread issued has retired once this fires
-        mbar_wait_bounded(bar(BAR_DRAIN), 0, &none, WAIT_LIMIT);
+        umma_commit(bar(C::BAR_DRAIN));   // everything this thread issued has retired once this fires
+        mbar_wait_bounded(bar(C::BAR_DRAIN), 0, &none, WAIT_LIMIT);
       }
     }
-  } else {
-    // ------------------------------------------------------------------ softmax: warps 2..5, one row per thread
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ softmax warpgroup x, one row per thread
+    const int x = (warp - 4) >> 2;
+    const int h = h0 + x;
     const int wq = warp & 3;            // a warp may only touch TMEM lanes 32*(warp % 4) ..
     const int row = wq * 32 + lane;
-    const uint32_t t_row = tmem + ((uint32_t)(wq * 32) << 16);
-    const uint32_t p_row = sP + row * 128;
+    const uint32_t t_s = tmem + ((uint32_t)(wq * 32) << 16) + x * 128;
+    const uint32_t t_o = tmem + ((uint32_t)(wq * 32) << 16) + (NT + x) * 128;
+    const uint32_t p_row = sP + x * TILE + row * 128;
     const uint32_t sw = (uint32_t)(row & 7);
     float m_ref = 0.f, l = 0.f;
     bool ok = true;
     for (int j = 0; j < n_tiles; ++j) {
-      ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(BAR_S), j & 1, abort_flag, WAIT_LIMIT));   // warp-uniform
+      ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_S + x), j & 1, abort_flag, WAIT_LIMIT));   // warp-uniform
       if (!ok) break;
       tc_fence_after();
       uint32_t s[4][32];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) tmem_ld_32x32(t_row + q * 32, s[q]);
+      for (int q = 0; q < 4; ++q) tmem_ld_32x32(t_s + q * 32, s[q]);
       tmem_wait_ld();
       if (j == n_tiles - 1) {   // diagonal tile: key column c is visible to row r iff c <= r
 #pragma unroll
@@ -199,16 +232,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         grow = true;
       }
       if (__any_sync(0xffffffffu, grow)) {
-        // the commit that signalled S_j also covers P V of tile j-1, so O is quiescent here
+        // S_x(j) was issued after P_x V of tile j-1, so the commit that signalled it covers that too: O_x is quiescent
         l *= alpha;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           uint32_t o[32];
-          tmem_ld_32x32(t_row + 128 + q * 32, o);
+          tmem_ld_32x32(t_o + q * 32, o);
           tmem_wait_ld();
 #pragma unroll
           for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-          tmem_st_32x32(t_row + 128 + q * 32, o);
+          tmem_st_32x32(t_o + q * 32, o);
         }
         tmem_wait_st();
       }
@@ -233,9 +266,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       l += sum;
       fence_async_smem();   // P was written through the generic proxy; the tensor core reads it through the async proxy
       tc_fence_before();
-      mbar_arrive(bar(BAR_P));
+      mbar_arrive(bar(C::BAR_P + x));
     }
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(BAR_O), 0, abort_flag, WAIT_LIMIT));
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_O + x), 0, abort_flag, WAIT_LIMIT));
     if (ok) {
       tc_fence_after();
       const float inv = 1.f / l;
@@ -244,7 +277,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         uint32_t o[32];
-        tmem_ld_32x32(t_row + 128 + q * 32, o);
+        tmem_ld_32x32(t_o + q * 32, o);
         tmem_wait_ld();
         if (valid) {
 #pragma unroll
@@ -267,7 +300,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, (int32_t)EARN_ERR_TIMEOUT);
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem, TMEM_COLS);
+    tmem_dealloc(tmem, C::TMEM_COLS);
   }
 }
 
@@ -298,6 +331,17 @@ bool make_map(CUtensorMap* map, const void* ptr, int heads, int total) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+template <int NT>
+cudaError_t launch_nt(const PrefillArgs& a, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                      const TcParams& p, cudaStream_t st) {
+  cudaError_t e = ensure_dynamic_smem<prefill_tc_kernel<NT>>(Cfg<NT>::SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  dim3 grid((a.max_seqlen + BM - 1) / BM, a.Hq / NT, a.batch);
+  prefill_tc_kernel<NT><<<grid, Cfg<NT>::THREADS, Cfg<NT>::SMEM_BYTES, st>>>(mq, mk, mv, p);
+  note_launch();
+  return cudaGetLastError();
+}
+
 }  // namespace
 
 bool prefill_tc_supported(const PrefillArgs& a, int total_tokens) {
@@ -309,16 +353,12 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int32_t* s
   if (!make_map(&mq, a.q, a.Hq, total_tokens) || !make_map(&mk, a.k, a.Hkv, total_tokens) ||
       !make_map(&mv, a.v, a.Hkv, total_tokens))
     return cudaErrorInvalidValue;
-  cudaError_t e = ensure_dynamic_smem<prefill_tc_kernel>(SMEM_BYTES);
-  if (e != cudaSuccess) return e;
   TcParams p{};
   p.o = a.o; p.lse = a.lse; p.cu_seqlens = a.cu_seqlens; p.status = status_word;
   p.Hq = a.Hq; p.g = a.Hq / a.Hkv; p.total = total_tokens;
   p.scale_log2 = a.scale * kLog2e;
-  dim3 grid((a.max_seqlen + BM - 1) / BM, a.Hq, a.batch);
-  prefill_tc_kernel<<<grid, 192, SMEM_BYTES, st>>>(mq, mk, mv, p);
-  note_launch();
-  return cudaGetLastError();
+  // two query heads of one kv head per CTA when the group size allows it
+  return (p.g % 2 == 0) ? launch_nt<2>(a, mq, mk, mv, p, st) : launch_nt<1>(a, mq, mk, mv, p, st);
 }
 
 }  // namespace earn
