@@ -23,7 +23,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2507_00715_b200 import workloads as wl  # noqa: E402
+from paper_2507_00715_b200 import replicas, workloads as wl  # noqa: E402
 
 METRIC = "EARN attn tokens/s/GPU (prefill+decode, 7B GQA)"
 UNIT = "tokens/s"
@@ -39,14 +39,33 @@ def read_peaks():
     return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
 
 
+KERNEL_SOURCES = {"prefill": "prefill_tc.cu", "compact": "compact.cu", "register": "register_mma.cu",
+                  "decode_compact": "decode_mma.cu", "decode_full": "decode_mma.cu"}
+
+
+def source_digest(fname: str) -> str:
+    import hashlib
+    with open(os.path.join(ROOT, "paper_2507_00715_b200", "csrc", fname), "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()[:12]
+
+
 def read_traffic(name: str) -> dict:
-    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) taken from the ncu captures
-    summarised under profiles/; {} when no capture of this workload has been recorded."""
-    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu captures summarised in
+    profiles/ncu_traffic.txt (lines: workload kind bytes source-file digest).  A figure is dropped when the
+    kernel's source file no longer matches the digest recorded with it."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.txt")
+    out = {}
     if not os.path.exists(path):
-        return {}
+        return out
     with open(path) as f:
-        return json.load(f).get(name, {})
+        for line in f:
+            parts = line.split("#")[0].split()
+            if len(parts) != 5 or parts[0] != name:
+                continue
+            _, kind, nbytes, fname, digest = parts
+            if source_digest(fname) == digest:
+                out[kind] = float(nbytes)
+    return out
 
 
 def workload_desc(w: wl.Workload) -> str:
@@ -461,7 +480,7 @@ def main():
         profile_one_kernel(w, dev, args.profile_kernel)
         return
 
-    job = GpuJob(w.replace(seed=w.seed + 1000 * rank) if rank else w, dev)
+    job = GpuJob(replicas.rank_workload(w, rank), dev)
     peaks = read_peaks()
 
     def barrier():
@@ -487,14 +506,10 @@ def main():
     barrier()
     launches = launches_per_step * args.steps
     clocks = sampler.stop() if sampler else None
-    elapsed = e0.elapsed_time(e1) * 1e-3
-    if dist is not None:
-        t = torch.tensor([elapsed], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed = float(t.item())
+    elapsed = replicas.max_over_ranks(e0.elapsed_time(e1) * 1e-3, dist, dev)
     assert job.ses.device_status() == 0, "a device-side wait timed out"
     t_step = elapsed / args.steps
-    value = world * tokens_per_step / t_step
+    value = replicas.job_throughput(tokens_per_step, world, t_step)
 
     # rooflines from the events recorded at the segment boundaries INSIDE the timed region
     alg = algorithmic(w)
@@ -516,8 +531,12 @@ def main():
         else:
             ach, peak, unit, bound = a["bytes"] / sec / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
             src = peaks["source"] + " (copy)"
+        if kind == "register_layer":
+            tr = traffic.get("compact", 0) + traffic.get("register", 0) if {"compact", "register"} <= set(traffic) else None
+        else:
+            tr = traffic.get(kind)
         rooflines[kind] = {"kernel": kind, "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
-                           "peak_source": src, "traffic": traffic.get(kind), "avg_launch_ms": sec * 1e3,
+                           "peak_source": src, "traffic": tr, "avg_launch_ms": sec * 1e3,
                            "launches_per_step": per_step, "share_of_step": share,
                            "algorithmic_flops_per_launch": a["flops"], "algorithmic_bytes_per_launch": a["bytes"]}
     roofline = max(rooflines.values(), key=lambda r: r["share_of_step"]) if rooflines else None
@@ -543,11 +562,7 @@ def main():
             job.step_e2e()
         a1.record()
         barrier()
-        te = a0.elapsed_time(a1) * 1e-3 / n_e2e
-        if dist is not None:
-            t = torch.tensor([te], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            te = float(t.item())
+        te = replicas.max_over_ranks(a0.elapsed_time(a1) * 1e-3 / n_e2e, dist, dev)
         e2e = {"value": world * tokens_per_step / te, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "ms_per_step": te * 1e3, "steps": n_e2e}
 
