@@ -144,6 +144,26 @@ earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* ba
                                const earn_cache_t* cache, void* o,
                                void* workspace, size_t workspace_bytes, earn_stream_t stream);
 
+/* earn_decode_attn for callers that cannot allocate device memory (the paper has no counterpart: this is a
+ * deployment variant of step 4, same arithmetic, same arguments minus the workspace).
+ * Meant for hosts that hand a plug-in its inputs and outputs and nothing else -- a serving framework that owns
+ * the whole memory pool, a latency-critical loop that cannot take cudaMalloc's device-wide synchronisation or
+ * its failure under memory pressure.  The scratch memory (status block, split tickets, split partials) lives
+ * in a fixed array of EARN_STATIC_SCRATCH_BYTES inside the library image; every GPU that loads the library
+ * holds that much until the process exits.  The call allocates nothing and frees nothing.
+ *   - A batch whose earn_workspace_bytes() exceeds EARN_STATIC_SCRATCH_BYTES is rejected with
+ *     EARN_ERR_WORKSPACE before anything is launched; use earn_decode_attn with your own workspace instead.
+ *   - The first call on each device looks up the array's device address (that device must be current, as for
+ *     every call); make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; each call clears
+ *     the part that must start at zero on `stream` before its kernel.  Two calls that overlap on the GPU (different
+ *     streams without an ordering between them) race on the array: serialise them. */
+#define EARN_STATIC_SCRATCH_BYTES (8u << 20)
+earn_status_t earn_decode_attn_static(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, int32_t step,
+                                      const void* q, const void* k_new, const void* v_new,
+                                      const void* k_full_or_null, const void* v_full_or_null,
+                                      const earn_cache_t* cache, void* o, earn_stream_t stream);
+
 /* Beam search bookkeeping between decode steps (Appendix A.3 uses beam search; the cache sharing is this
  * library's design): before step `step` (>= 2), beam j continues the history of beam parent[j] (an index in
  * [0,W) within its own sequence).  No K/V moves: lineage_out[j][t] = lineage_in[b*W+parent[j]][t] for

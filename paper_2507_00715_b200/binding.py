@@ -55,6 +55,9 @@ SYMBOLS = {
     "earn_decode_attn": (C.c_int, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32, C.c_int32, C.c_void_p,
                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(EarnCache), C.c_void_p,
                                    C.c_void_p, C.c_size_t, C.c_void_p]),
+    "earn_decode_attn_static": (C.c_int, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32, C.c_int32, C.c_void_p,
+                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(EarnCache), C.c_void_p,
+                                          C.c_void_p]),
     "earn_beam_reparent": (C.c_int, [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.c_void_p]),
     "earn_launch_count": (C.c_uint64, []),
@@ -188,6 +191,18 @@ def earn_decode_attn(model, batch: Batch, layer, step, q, k_new, v_new, cache: E
     _check(lib().earn_decode_attn(C.byref(model), C.byref(batch.c), layer, step, _ptr(q), _ptr(k_new), _ptr(v_new),
                                   _ptr(k_full), _ptr(v_full), C.byref(cache), _ptr(o), p, n, _stream()),
            "earn_decode_attn")
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def earn_decode_attn_static(model, batch: Batch, layer, step, q, k_new, v_new, cache: EarnCache, o, k_full=None,
+                            v_full=None) -> None:
+    """earn_decode_attn without a workspace argument: the library's built-in scratch array is used, so the
+    caller needs no device allocation of its own (batches that need more than STATIC_SCRATCH_BYTES raise)."""
+    _check(lib().earn_decode_attn_static(C.byref(model), C.byref(batch.c), layer, step, _ptr(q), _ptr(k_new),
+                                         _ptr(v_new), _ptr(k_full), _ptr(v_full), C.byref(cache), _ptr(o), _stream()),
+           "earn_decode_attn_static")
 
 
 def earn_beam_reparent(batch: int, beams: int, max_new: int, step: int, parent, lineage_in, lineage_out) -> None:
