@@ -57,9 +57,7 @@ extern "C" earn_status_t earn_decode_attn_static(const earn_model_t* model, cons
   if (scratch_address(&scratch) != cudaSuccess) return EARN_ERR_CUDA;
   // The array keeps whatever the previous call left.  The status block and the tickets must read zero when the
   // kernel starts; the partials behind them are always written before they are read.
-  const DecodePlan plan = make_decode_plan(*model, *batch, cache->beams, batch->max_seqlen);
-  size_t head = (size_t)kStatusBytes +
-                (sizeof(int32_t) * (size_t)batch->batch * model->n_kv_heads * plan.row_tiles + 255) / 256 * 256;
+  size_t head = workspace_head_bytes(*model, *batch, cache->beams);
   if (head > need) head = need;
   if (cudaMemsetAsync(scratch, 0, head, (cudaStream_t)stream) != cudaSuccess) return EARN_ERR_CUDA;
   return earn_decode_attn(model, batch, layer, step, q, k_new, v_new, k_full_or_null, v_full_or_null, cache, o, scratch,

@@ -78,11 +78,20 @@ static size_t ticket_bytes(const earn_model_t& m, const earn_batch_t& b, const D
   return round_up(sizeof(int32_t) * (size_t)b.batch * m.n_kv_heads * p.row_tiles, 256);
 }
 
+size_t prefill_plan_bytes(const earn_batch_t& b) {
+  if (b.batch <= 0 || b.cu_seqlens_host == nullptr) return 0;
+  return round_up(sizeof(int4) * (size_t)prefill_plan_entries(b), 256);
+}
+
+size_t workspace_head_bytes(const earn_model_t& m, const earn_batch_t& b, int beams) {
+  return kStatusBytes + prefill_plan_bytes(b) + ticket_bytes(m, b, make_decode_plan(m, b, beams, b.max_seqlen));
+}
+
 static size_t workspace_need(const earn_model_t* m, const earn_batch_t* b, int beams) {
   DecodePlan full = make_decode_plan(*m, *b, beams, b->max_seqlen);
   DecodePlan reg = make_decode_plan(*m, *b, beams, b->n_head_reg + b->n_tail_reg);
   size_t f = decode_partial_floats(*m, *b, full), r = decode_partial_floats(*m, *b, reg);
-  return kStatusBytes + ticket_bytes(*m, *b, full) + round_up(sizeof(float) * (f > r ? f : r), 256) + 256;
+  return workspace_head_bytes(*m, *b, beams) + round_up(sizeof(float) * (f > r ? f : r), 256) + 256;
 }
 
 static earn_status_t check_cache_shared(const earn_model_t* m, const earn_batch_t* b, const earn_cache_t* c) {
@@ -130,7 +139,7 @@ const char* earn_status_string(earn_status_t s) {
 }
 
 size_t earn_workspace_bytes(const earn_model_t* model, const earn_batch_t* batch, int32_t beams) {
-  if (check_model(model) != EARN_OK || batch == nullptr || beams < 1) return kStatusBytes;
+  if (check_model(model) != EARN_OK || check_batch(batch) != EARN_OK || beams < 1) return kStatusBytes;
   return workspace_need(model, batch, beams);
 }
 
@@ -168,9 +177,10 @@ earn_status_t earn_prefill_attn(const earn_model_t* model, const earn_batch_t* b
   a.Hq = model->n_q_heads; a.Hkv = model->n_kv_heads; a.D = model->head_dim; a.dtype = model->dtype;
   a.scale = scale_of(model);
   if (prefill_tc_supported(a, batch->total_tokens)) {
-    if (!aligned16(workspace)) return EARN_ERR_WORKSPACE;
-    return launch_prefill_tc(a, batch->total_tokens, reinterpret_cast<int32_t*>(workspace), (cudaStream_t)stream) ==
-                   cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+    if (!aligned16(workspace) || workspace_bytes < kStatusBytes + prefill_plan_bytes(*batch)) return EARN_ERR_WORKSPACE;
+    return launch_prefill_tc(a, batch->total_tokens, prefill_plan_entries(*batch),
+                             reinterpret_cast<char*>(workspace) + kStatusBytes, reinterpret_cast<int32_t*>(workspace),
+                             (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
   }
   return launch_prefill_simt(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
 }
@@ -264,8 +274,9 @@ earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* ba
   a.k_priv = cache->k_priv; a.v_priv = cache->v_priv; a.lineage = cache->lineage;
   a.plan = make_decode_plan(*model, *batch, cache->beams,
                             early ? batch->max_seqlen : batch->n_head_reg + batch->n_tail_reg);
-  a.tickets = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(workspace) + kStatusBytes);
-  a.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) + kStatusBytes + ticket_bytes(*model, *batch, a.plan));
+  const size_t tickets_at = kStatusBytes + prefill_plan_bytes(*batch);
+  a.tickets = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(workspace) + tickets_at);
+  a.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) + tickets_at + ticket_bytes(*model, *batch, a.plan));
   a.part_lse = a.part_o + (size_t)batch->batch * model->n_kv_heads * a.plan.n_splits * a.plan.rows_pad * model->head_dim;
   a.batch = batch->batch; a.beams = cache->beams; a.max_new = cache->max_new; a.step = step;
   a.Hq = model->n_q_heads; a.Hkv = model->n_kv_heads; a.D = model->head_dim; a.dtype = model->dtype;

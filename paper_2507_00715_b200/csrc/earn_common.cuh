@@ -48,6 +48,11 @@ constexpr int kDecodeRows = 16;
 DecodePlan make_decode_plan(const earn_model_t& m, const earn_batch_t& b, int beams, int max_shared_len);
 size_t decode_partial_floats(const earn_model_t& m, const earn_batch_t& b, const DecodePlan& p);
 
+// Workspace layout: status block | prefill plan | split-decode tickets | split-decode partials.
+size_t prefill_plan_bytes(const earn_batch_t& b);
+// status block + plan + tickets: the part of the workspace that must read zero before the first call
+size_t workspace_head_bytes(const earn_model_t& m, const earn_batch_t& b, int beams);
+
 void note_launch(int n = 1);   // host-side count of kernels launched by this library
 
 // Opt a kernel in to `bytes` of dynamic shared memory, once per device (the attribute call is not free).
@@ -75,7 +80,10 @@ struct PrefillArgs {
 cudaError_t launch_prefill_simt(const PrefillArgs& a, cudaStream_t st);
 // tensor-core path (bf16, head_dim 128); status_word receives EARN_ERR_TIMEOUT if a bounded wait runs out
 bool prefill_tc_supported(const PrefillArgs& a, int total_tokens);
-cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int32_t* status_word, cudaStream_t st);
+int prefill_plan_entries(const earn_batch_t& b);   // (sequence, 128-row query tile) pairs of the batch
+// plan: device scratch of 16 bytes per plan entry, filled by a planning kernel launched ahead of the main one
+cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int plan_entries, void* plan, int32_t* status_word,
+                              cudaStream_t st);
 
 struct RegisterArgs {
   const void* q_reg;

@@ -1,13 +1,21 @@
 // Full causal prefill attention (Eq. 3 + causal mask, layers l < k) on the Blackwell tensor cores.
 // bf16 Q/K/V, head_dim 128, fp32 logits / softmax / accumulation, bf16 output.
 //
-// One CTA = 128 query rows of NT query heads that share a kv head (NT = 2 when the GQA group size is
-// even, else 1): NT "M-tiles" with the same rows and the same key range, so they share every K/V tile
-// and finish together.  Per 128-key tile:
+// Work item = 128 query rows of NT query heads that share a kv head (NT = 2 when the GQA group size is
+// even, else 1): NT "M-tiles" with the same rows and the same key range, so they share every K/V tile.
+// A small planning kernel lists the (sequence, query tile) pairs of the batch, longest key range first;
+// the main kernel is persistent (one CTA per SM) and CTA c takes items c, c + gridDim, ... of that list,
+// so every SM gets the same mix of long and short items and the pipeline below never drains between items.
+//
 //   warp 0     TMA: K and V tiles -> shared memory (128-byte swizzle), a ring of 32 KB entries K0 V0 K1 V1 ..
-//   warp 1     one thread issues tcgen05.mma: S_x = Q_x K^T into tensor memory, later O_x += P_x V
-//   warps 4..  one softmax warpgroup per M-tile, one query row per thread: read S_x from TMEM, online softmax
-//              in the log2 domain, write P_x as bf16 into swizzled shared memory
+//              that runs on across item boundaries
+//   warp 2     TMA: the Q tiles of the next item, as soon as the last S of the current item has read them
+//   warp 1     one thread issues tcgen05.mma: S_x = Q_x K^T into tensor memory, O_x += P_x V with P_x read
+//              from tensor memory; after the last P V of an item it goes straight on to the first S of the next
+//   warps 4..  one softmax warpgroup per M-tile, one query row per thread: S_x from TMEM in 32-column chunks
+//              (one pass for the row maximum, one for the exponentials), online softmax in the log2 domain,
+//              P_x written back as bf16 over the columns of S_x it has already consumed; the same warps
+//              normalise and store O_x when the item ends, while the tensor core already works on the next item
 // With two M-tiles the tensor core works on one while the other is in its softmax (S_A, S_B, O_A, O_B fill
 // the 512 TMEM columns).  The running output stays in TMEM.  The softmax reference maximum is only raised
 // when the row maximum grows by more than 2^8; then the owning warp rescales its 32 rows of O in TMEM.
@@ -32,44 +40,70 @@ constexpr float RESCALE_THRESHOLD = 8.f;           // log2 units
 
 template <int NT>
 struct Cfg {
-  static constexpr int NSTAGE = NT == 1 ? 4 : 3;            // ring entries (K and V tiles alternate)
+  static constexpr int NSTAGE = NT == 1 ? 6 : 5;            // ring entries (K and V tiles alternate)
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_RING = OFF_Q + NT * TILE;
-  static constexpr int OFF_P = OFF_RING + NSTAGE * TILE;
-  static constexpr int OFF_BAR = OFF_P + NT * TILE;
-  static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;   // + alignment slack
-  static constexpr int TMEM_COLS = NT * 256;                // S_x at x*128, O_x at (NT + x)*128
+  static constexpr int OFF_BAR = OFF_RING + NSTAGE * TILE;
+  static constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;   // + alignment slack
+  static constexpr int TMEM_COLS = NT * 256;                // S_x (and P_x over it) at x*128, O_x at (NT + x)*128
   static constexpr int THREADS = 32 * (4 + 4 * NT);
   // barriers
-  static constexpr int BAR_Q = 0, BAR_FULL = 1, BAR_EMPTY = BAR_FULL + NSTAGE, BAR_S = BAR_EMPTY + NSTAGE,
-                       BAR_P = BAR_S + NT, BAR_O = BAR_P + NT, BAR_DRAIN = BAR_O + NT, N_BARS = BAR_DRAIN + 1;
+  static constexpr int BAR_FULL = 0, BAR_EMPTY = BAR_FULL + NSTAGE, BAR_QFULL = BAR_EMPTY + NSTAGE,
+                       BAR_QFREE = BAR_QFULL + NT, BAR_S = BAR_QFREE + NT, BAR_P = BAR_S + NT, BAR_O = BAR_P + NT,
+                       BAR_DRAIN = BAR_O + NT, N_BARS = BAR_DRAIN + 1;
+  static_assert(8 * N_BARS + 16 <= 512, "barrier block");
 };
 
 struct TcParams {
   void* o;
   float* lse;
-  const int32_t* cu_seqlens;
+  const int4* plan;        // one entry per (sequence, query tile): {first global row, rows of the sequence from there, tile index, sequence}
   int32_t* status;
-  int Hq, g, total;
+  int Hq, g, total, n_items, n_hp;   // n_hp = Hq / NT work items per plan entry
   float scale_log2;
 };
 
+struct Item {
+  int row0;      // global row of the first query of the tile
+  int rows;      // rows of the sequence from there on (>= 1); the tile holds min(rows, 128) valid rows
+  int n_tiles;   // key tiles 0 .. diagonal
+  int key0;      // global row of the sequence's first key
+  int h0;        // first query head
+};
+
+__device__ __forceinline__ Item load_item(const TcParams& p, int i, int NT) {
+  const int e = i / p.n_hp, hp = i - e * p.n_hp;
+  const int4 t = __ldg(p.plan + e);
+  Item it;
+  it.row0 = t.x; it.rows = t.y; it.n_tiles = t.z + 1; it.key0 = t.x - t.z * BM; it.h0 = hp * NT;
+  return it;
+}
+
+// ---- packed fp32 pairs (one instruction for two lanes of the row) and three-input max
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ void fma2(float& d0, float& d1, float a0, float a1, float b, float c) {   // d = a * b + c
+  asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %5};\n\t"
+      "fma.rn.ftz.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b), "f"(c));
+}
+__device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {   // d += a
+  asm("{\n\t.reg .b64 ra, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rd, {%0, %1};\n\tadd.rn.ftz.f32x2 rd, rd, ra;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
+}
 template <int NT>
 __global__ void __launch_bounds__(Cfg<NT>::THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, TcParams p) {
   using C = Cfg<NT>;
-  const int b = blockIdx.z, h0 = blockIdx.y * NT;
-  const int lo = p.cu_seqlens[b], L = p.cu_seqlens[b + 1] - lo;
-  const int q0 = ((int)gridDim.x - 1 - (int)blockIdx.x) * BM;   // longest tiles first
-  if (q0 >= L) return;
-  const int n_tiles = q0 / BN + 1;                                // causal: key tiles 0 .. diagonal
-  const int kvh = h0 / p.g;
-
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;    // swizzled tiles need 1024-byte alignment
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t sQ = base + C::OFF_Q, sRing = base + C::OFF_RING, sP = base + C::OFF_P;
+  const uint32_t sQ = base + C::OFF_Q, sRing = base + C::OFF_RING;
   const uint32_t bars = base + C::OFF_BAR;
   auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + C::OFF_BAR + 8 * C::N_BARS);
@@ -77,12 +111,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    mbar_init(bar(C::BAR_Q), 1);
     for (int s = 0; s < C::NSTAGE; ++s) {
       mbar_init(bar(C::BAR_FULL + s), 1);
       mbar_init(bar(C::BAR_EMPTY + s), 1);
     }
     for (int x = 0; x < NT; ++x) {
+      mbar_init(bar(C::BAR_QFULL + x), 1);
+      mbar_init(bar(C::BAR_QFREE + x), 1);
       mbar_init(bar(C::BAR_S + x), 1);
       mbar_init(bar(C::BAR_P + x), 128);
       mbar_init(bar(C::BAR_O + x), 1);
@@ -102,45 +137,68 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const int n_entries = 2 * n_tiles;   // ring entries: K_0 V_0 K_1 V_1 ...
+  const int first = blockIdx.x, stride = gridDim.x;   // this CTA's items: first, first + stride, ...
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ TMA producer: K/V ring
     if (lane == 0) {
-      mbar_expect_tx(bar(C::BAR_Q), NT * TILE);
-      for (int x = 0; x < NT; ++x) {
-        tma_load_3d(sQ + x * TILE, &map_q, bar(C::BAR_Q), 0, h0 + x, lo + q0);
-        tma_load_3d(sQ + x * TILE + HALF, &map_q, bar(C::BAR_Q), 64, h0 + x, lo + q0);
-      }
-      int issued = 0;
-      for (int e = 0; e < n_entries; ++e) {
-        const int st = e % C::NSTAGE;
-        if (e >= C::NSTAGE &&
-            !mbar_wait_bounded(bar(C::BAR_EMPTY + st), ((e / C::NSTAGE) - 1) & 1, abort_flag, WAIT_LIMIT))
-          break;
-        const CUtensorMap* map = (e & 1) ? &map_v : &map_k;
-        mbar_expect_tx(bar(C::BAR_FULL + st), TILE);
-        tma_load_3d(sRing + st * TILE, map, bar(C::BAR_FULL + st), 0, kvh, lo + (e >> 1) * BN);
-        tma_load_3d(sRing + st * TILE + HALF, map, bar(C::BAR_FULL + st), 64, kvh, lo + (e >> 1) * BN);
-        issued = e + 1;
+      int e = 0;   // ring entries issued so far, over all items
+      bool ok = true;
+      for (int i = first; i < p.n_items && ok; i += stride) {
+        const Item it = load_item(p, i, NT);
+        const int kvh = it.h0 / p.g;
+        for (int t = 0; t < 2 * it.n_tiles; ++t, ++e) {
+          const int st = e % C::NSTAGE;
+          if (e >= C::NSTAGE &&
+              !mbar_wait_bounded(bar(C::BAR_EMPTY + st), ((e / C::NSTAGE) - 1) & 1, abort_flag, WAIT_LIMIT)) {
+            ok = false;
+            break;
+          }
+          const CUtensorMap* map = (t & 1) ? &map_v : &map_k;
+          mbar_expect_tx(bar(C::BAR_FULL + st), TILE);
+          tma_load_3d(sRing + st * TILE, map, bar(C::BAR_FULL + st), 0, kvh, it.key0 + (t >> 1) * BN);
+          tma_load_3d(sRing + st * TILE + HALF, map, bar(C::BAR_FULL + st), 64, kvh, it.key0 + (t >> 1) * BN);
+        }
       }
       if (*abort_flag) {
         // let the copies already in flight land before the CTA gives its shared memory back
         int none = 0;
-        mbar_wait_bounded(bar(C::BAR_Q), 0, &none, WAIT_LIMIT);
-        for (int e = max(issued - C::NSTAGE, 0); e < issued; ++e)
-          mbar_wait_bounded(bar(C::BAR_FULL + e % C::NSTAGE), (e / C::NSTAGE) & 1, &none, WAIT_LIMIT);
+        for (int f = max(e - C::NSTAGE, 0); f < e; ++f)
+          mbar_wait_bounded(bar(C::BAR_FULL + f % C::NSTAGE), (f / C::NSTAGE) & 1, &none, WAIT_LIMIT);
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ TMA producer: Q tiles
+    if (lane == 0) {
+      int n = 0;   // items loaded so far
+      bool ok = true;
+      for (int i = first; i < p.n_items && ok; i += stride, ++n) {
+        const Item it = load_item(p, i, NT);
+        for (int x = 0; x < NT; ++x) {
+          if (n > 0 && !mbar_wait_bounded(bar(C::BAR_QFREE + x), (n - 1) & 1, abort_flag, WAIT_LIMIT)) {
+            ok = false;
+            break;
+          }
+          mbar_expect_tx(bar(C::BAR_QFULL + x), TILE);
+          tma_load_3d(sQ + x * TILE, &map_q, bar(C::BAR_QFULL + x), 0, it.h0 + x, it.row0);
+          tma_load_3d(sQ + x * TILE + HALF, &map_q, bar(C::BAR_QFULL + x), 64, it.h0 + x, it.row0);
+        }
+      }
+      if (*abort_flag && n > 0) {
+        int none = 0;
+        for (int x = 0; x < NT; ++x) mbar_wait_bounded(bar(C::BAR_QFULL + x), (n - 1) & 1, &none, WAIT_LIMIT);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc_s = idesc_bf16_f32(BM, BN, 0, 0);   // Q (K-major) x K^T (K-major)
-      constexpr uint32_t idesc_o = idesc_bf16_f32(BM, HD, 0, 1);   // P (K-major) x V (MN-major)
+      constexpr uint32_t idesc_o = idesc_bf16_f32(BM, HD, 0, 1);   // P (TMEM) x V (MN-major)
       auto wait_full = [&](int e) {
         return mbar_wait_bounded(bar(C::BAR_FULL + e % C::NSTAGE), (e / C::NSTAGE) & 1, abort_flag, WAIT_LIMIT);
       };
-      auto issue_s = [&](int x, int e) {   // S_x = Q_x K^T with the K tile of ring entry e
+      // S_x = Q_x K^T with the K tile of ring entry e; `last` = no later S of this item reads Q_x
+      auto issue_s = [&](int x, int e, bool last) {
         const uint32_t sK = sRing + (e % C::NSTAGE) * TILE;
 #pragma unroll
         for (int kk = 0; kk < HD / 16; ++kk) {
@@ -149,39 +207,65 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                   idesc_s, kk > 0);
         }
         umma_commit(bar(C::BAR_S + x));
+        if (last) umma_commit(bar(C::BAR_QFREE + x));
         if (x == NT - 1) umma_commit(bar(C::BAR_EMPTY + e % C::NSTAGE));   // K tile free once the last S has read it
       };
-      auto issue_pv = [&](int x, int e, bool first) {   // O_x (+)= P_x V with the V tile of ring entry e
+      // O_x (+)= P_x V with P_x in tensor memory (bf16 pairs over the first 64 columns of S_x) and the V tile of entry e
+      auto issue_pv = [&](int x, int e, bool first_tile) {
         const uint32_t sV = sRing + (e % C::NSTAGE) * TILE;
 #pragma unroll
-        for (int kk = 0; kk < BN / 16; ++kk) {
-          const uint32_t offp = (kk >> 2) * HALF + (kk & 3) * 32;
-          umma_ss(tmem + (NT + x) * 128, smem_desc_sw128(sP + x * TILE + offp, 16, 1024),
-                  smem_desc_sw128(sV + kk * 2048, HALF, 1024), idesc_o, (!first || kk > 0) ? 1u : 0u);
-        }
+        for (int kk = 0; kk < BN / 16; ++kk)
+          umma_ts(tmem + (NT + x) * 128, tmem + x * 128 + kk * 8, smem_desc_sw128(sV + kk * 2048, HALF, 1024), idesc_o,
+                  (!first_tile || kk > 0) ? 1u : 0u);
         if (x == NT - 1) umma_commit(bar(C::BAR_EMPTY + e % C::NSTAGE));   // V tile free once the last P V has read it
       };
-      bool ok = mbar_wait_bounded(bar(C::BAR_Q), 0, abort_flag, WAIT_LIMIT) && wait_full(0);
+      int eb = 0;       // ring entry of the current item's K_0
+      int n_item = 0;   // items started so far
+      int n_p[NT];      // P_x phases consumed so far
+      for (int x = 0; x < NT; ++x) n_p[x] = 0;
+      bool ok = first < p.n_items;
+      Item cur{};
       if (ok) {
-        tc_fence_after();
-        for (int x = 0; x < NT; ++x) issue_s(x, 0);
-      }
-      for (int j = 0; j < n_tiles && ok; ++j) {
+        cur = load_item(p, first, NT);
         for (int x = 0; x < NT && ok; ++x) {
-          ok = mbar_wait_bounded(bar(C::BAR_P + x), j & 1, abort_flag, WAIT_LIMIT);   // P_x(j) written, S_x free
-          if (ok && x == 0) ok = wait_full(2 * j + 1);
+          ok = mbar_wait_bounded(bar(C::BAR_QFULL + x), 0, abort_flag, WAIT_LIMIT) && (x > 0 || wait_full(0));
           if (!ok) break;
           tc_fence_after();
-          issue_pv(x, 2 * j + 1, j == 0);
-          if (j == n_tiles - 1) {
-            umma_commit(bar(C::BAR_O + x));
-          } else {
-            if (x == 0) ok = wait_full(2 * j + 2);
+          issue_s(x, 0, cur.n_tiles == 1);
+        }
+      }
+      for (int i = first; i < p.n_items && ok; i += stride, ++n_item) {
+        const bool has_next = i + stride < p.n_items;
+        Item nxt{};
+        if (has_next) nxt = load_item(p, i + stride, NT);
+        const int n = cur.n_tiles;
+        for (int j = 0; j < n && ok; ++j) {
+          for (int x = 0; x < NT && ok; ++x) {
+            ok = mbar_wait_bounded(bar(C::BAR_P + x), n_p[x] & 1, abort_flag, WAIT_LIMIT);   // P_x(j) written, S_x consumed
+            ++n_p[x];
+            if (ok && x == 0) ok = wait_full(eb + 2 * j + 1);
             if (!ok) break;
             tc_fence_after();
-            issue_s(x, 2 * j + 2);
+            issue_pv(x, eb + 2 * j + 1, j == 0);
+            if (j < n - 1) {
+              if (x == 0) ok = wait_full(eb + 2 * j + 2);
+              if (!ok) break;
+              tc_fence_after();
+              issue_s(x, eb + 2 * j + 2, j + 1 == n - 1);
+            } else {
+              umma_commit(bar(C::BAR_O + x));
+              if (has_next) {   // straight on to the next item: its Q_x and first K tile are on their way already
+                ok = mbar_wait_bounded(bar(C::BAR_QFULL + x), (n_item + 1) & 1, abort_flag, WAIT_LIMIT);
+                if (ok && x == 0) ok = wait_full(eb + 2 * n);
+                if (!ok) break;
+                tc_fence_after();
+                issue_s(x, eb + 2 * n, nxt.n_tiles == 1);
+              }
+            }
           }
         }
+        eb += 2 * n;
+        cur = nxt;
       }
       if (*abort_flag) {
         int none = 0;
@@ -192,106 +276,136 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ softmax warpgroup x, one row per thread
     const int x = (warp - 4) >> 2;
-    const int h = h0 + x;
     const int wq = warp & 3;            // a warp may only touch TMEM lanes 32*(warp % 4) ..
     const int row = wq * 32 + lane;
-    const uint32_t t_s = tmem + ((uint32_t)(wq * 32) << 16) + x * 128;
+    const uint32_t t_s = tmem + ((uint32_t)(wq * 32) << 16) + x * 128;   // S_x; P_x goes over its first 64 columns
     const uint32_t t_o = tmem + ((uint32_t)(wq * 32) << 16) + (NT + x) * 128;
-    const uint32_t p_row = sP + x * TILE + row * 128;
-    const uint32_t sw = (uint32_t)(row & 7);
-    float m_ref = 0.f, l = 0.f;
+    const float sl2 = p.scale_log2;
+    int n_s = 0, n_item = 0;
     bool ok = true;
-    for (int j = 0; j < n_tiles; ++j) {
-      ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_S + x), j & 1, abort_flag, WAIT_LIMIT));   // warp-uniform
-      if (!ok) break;
-      tc_fence_after();
-      uint32_t s[4][32];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) tmem_ld_32x32(t_s + q * 32, s[q]);
-      tmem_wait_ld();
-      if (j == n_tiles - 1) {   // diagonal tile: key column c is visible to row r iff c <= r
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-#pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if (q * 32 + c > row) s[q][c] = 0xff800000u;   // -inf
-      }
-      float mx = -INFINITY;
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-#pragma unroll
-        for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(s[q][c]));
-      mx *= p.scale_log2;
-      float alpha = 1.f;
-      bool grow = false;
-      if (j == 0) {
-        m_ref = mx;
-      } else if (mx > m_ref + RESCALE_THRESHOLD) {
-        alpha = ex2(m_ref - mx);
-        m_ref = mx;
-        grow = true;
-      }
-      if (__any_sync(0xffffffffu, grow)) {
-        // S_x(j) was issued after P_x V of tile j-1, so the commit that signalled it covers that too: O_x is quiescent
-        l *= alpha;
+    for (int i = first; i < p.n_items && ok; i += stride, ++n_item) {
+      const Item it = load_item(p, i, NT);
+      const int h = it.h0 + x;
+      float m_ref = 0.f, l0 = 0.f, l1 = 0.f;
+      for (int j = 0; j < it.n_tiles; ++j, ++n_s) {
+        ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_S + x), n_s & 1, abort_flag, WAIT_LIMIT));   // warp-uniform
+        if (!ok) break;
+        tc_fence_after();
+        const bool diag = j == it.n_tiles - 1;        // key column c of this tile is visible to row r iff c <= r
+        const int n_chunks = diag ? wq + 1 : 4;       // 32-column chunks with a visible key for this warp's rows
+        uint32_t a[32], b[32];
+        // ---- pass 1: row maximum
+        float mx = -INFINITY;
+        tmem_ld_32x32(t_s, a);
+        tmem_wait_ld(a);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          uint32_t o[32];
-          tmem_ld_32x32(t_o + q * 32, o);
-          tmem_wait_ld();
+          if (q < n_chunks) {
+            uint32_t(&cur)[32] = (q & 1) ? b : a;
+            uint32_t(&nxt)[32] = (q & 1) ? a : b;
+            if (q + 1 < n_chunks) tmem_ld_32x32(t_s + (q + 1) * 32, nxt);
+            if (diag && q == wq) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-          tmem_st_32x32(t_o + q * 32, o);
+              for (int c = 0; c < 32; ++c)
+                if (c > lane) cur[c] = 0xff800000u;   // -inf
+            }
+#pragma unroll
+            for (int c = 0; c < 32; c += 2) mx = max3(mx, __uint_as_float(cur[c]), __uint_as_float(cur[c + 1]));
+            if (q + 1 < n_chunks) tmem_wait_ld(nxt);
+          }
+        }
+        mx *= sl2;
+        float alpha = 1.f;
+        bool grow = false;
+        if (j == 0) {
+          m_ref = mx;
+        } else if (mx > m_ref + RESCALE_THRESHOLD) {
+          alpha = ex2(m_ref - mx);
+          m_ref = mx;
+          grow = true;
+        }
+        if (__any_sync(0xffffffffu, grow)) {
+          // S_x(j) was issued after P_x V of tile j-1, so the commit that signalled it covers that too: O_x is quiescent
+          l0 *= alpha;
+          l1 *= alpha;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            tmem_ld_32x32(t_o + q * 32, a);
+            tmem_wait_ld(a);
+#pragma unroll
+            for (int c = 0; c < 32; ++c) a[c] = __float_as_uint(__uint_as_float(a[c]) * alpha);
+            tmem_st_32x32(t_o + q * 32, a);
+          }
+        }
+        // ---- pass 2: P = 2^(S * scale - m_ref) as bf16 pairs, written over the consumed columns of S_x
+        const float neg_m = -m_ref;
+        tmem_ld_32x32(t_s, a);
+        tmem_wait_ld(a);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          uint32_t pk[16];
+          if (q < n_chunks) {
+            uint32_t(&cur)[32] = (q & 1) ? b : a;
+            uint32_t(&nxt)[32] = (q & 1) ? a : b;
+            if (q + 1 < n_chunks) tmem_ld_32x32(t_s + (q + 1) * 32, nxt);
+            if (diag && q == wq) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c)
+                if (c > lane) cur[c] = 0xff800000u;
+            }
+#pragma unroll
+            for (int c = 0; c < 32; c += 2) {
+              float e0, e1;
+              fma2(e0, e1, __uint_as_float(cur[c]), __uint_as_float(cur[c + 1]), sl2, neg_m);
+              e0 = ex2(e0);
+              e1 = ex2(e1);
+              add2(l0, l1, e0, e1);
+              pk[c >> 1] = pack_bf16(e0, e1);
+            }
+            tmem_st_32x16(t_s + q * 16, pk);
+            if (q + 1 < n_chunks) tmem_wait_ld(nxt);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 16; ++c) pk[c] = 0u;
+            tmem_st_32x16(t_s + q * 16, pk);
+          }
         }
         tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(C::BAR_P + x));
       }
-      float sum = 0.f;
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-#pragma unroll
-        for (int c8 = 0; c8 < 4; ++c8) {
-          float e[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            e[i] = ex2(fmaf(__uint_as_float(s[q][c8 * 8 + i]), p.scale_log2, -m_ref));
-            sum += e[i];
-          }
-          const uint32_t chunk = (uint32_t)((q & 1) * 4 + c8);
-          const uint32_t addr = p_row + (q >> 1) * HALF + ((chunk ^ sw) << 4);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(pack_bf16(e[0], e[1])),
-                       "r"(pack_bf16(e[2], e[3])), "r"(pack_bf16(e[4], e[5])), "r"(pack_bf16(e[6], e[7]))
-                       : "memory");
-        }
-      }
-      l += sum;
-      fence_async_smem();   // P was written through the generic proxy; the tensor core reads it through the async proxy
-      tc_fence_before();
-      mbar_arrive(bar(C::BAR_P + x));
-    }
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_O + x), 0, abort_flag, WAIT_LIMIT));
-    if (ok) {
+      if (!ok) break;
+      // ---- end of the item: O_x / l -> global memory (the tensor core is already on the next item's S)
+      ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_O + x), n_item & 1, abort_flag, WAIT_LIMIT));
+      if (!ok) break;
       tc_fence_after();
+      const float l = l0 + l1;
       const float inv = 1.f / l;
-      const bool valid = q0 + row < L;
-      __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) + ((int64_t)(lo + q0 + row) * p.Hq + h) * HD;
+      const bool valid = row < it.rows;
+      __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) + ((int64_t)(it.row0 + row) * p.Hq + h) * HD;
+      uint32_t a[32], b[32];
+      tmem_ld_32x32(t_o, a);
+      tmem_wait_ld(a);
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        uint32_t o[32];
-        tmem_ld_32x32(t_o + q * 32, o);
-        tmem_wait_ld();
+        uint32_t(&cur)[32] = (q & 1) ? b : a;
+        uint32_t(&nxt)[32] = (q & 1) ? a : b;
+        if (q + 1 < 4) tmem_ld_32x32(t_o + (q + 1) * 32, nxt);
         if (valid) {
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             uint4 w;
-            w.x = pack_bf16(__uint_as_float(o[c * 8 + 0]) * inv, __uint_as_float(o[c * 8 + 1]) * inv);
-            w.y = pack_bf16(__uint_as_float(o[c * 8 + 2]) * inv, __uint_as_float(o[c * 8 + 3]) * inv);
-            w.z = pack_bf16(__uint_as_float(o[c * 8 + 4]) * inv, __uint_as_float(o[c * 8 + 5]) * inv);
-            w.w = pack_bf16(__uint_as_float(o[c * 8 + 6]) * inv, __uint_as_float(o[c * 8 + 7]) * inv);
+            w.x = pack_bf16(__uint_as_float(cur[c * 8 + 0]) * inv, __uint_as_float(cur[c * 8 + 1]) * inv);
+            w.y = pack_bf16(__uint_as_float(cur[c * 8 + 2]) * inv, __uint_as_float(cur[c * 8 + 3]) * inv);
+            w.z = pack_bf16(__uint_as_float(cur[c * 8 + 4]) * inv, __uint_as_float(cur[c * 8 + 5]) * inv);
+            w.w = pack_bf16(__uint_as_float(cur[c * 8 + 6]) * inv, __uint_as_float(cur[c * 8 + 7]) * inv);
             *reinterpret_cast<uint4*>(orow + q * 32 + c * 8) = w;
           }
         }
+        if (q + 1 < 4) tmem_wait_ld(nxt);
       }
-      if (valid && p.lse != nullptr) p.lse[(int64_t)h * p.total + lo + q0 + row] = (m_ref + log2f(l)) * kLn2;
+      if (valid && p.lse != nullptr) p.lse[(int64_t)h * p.total + it.row0 + row] = (m_ref + log2f(l)) * kLn2;
+      tc_fence_before();   // the next item's first P V overwrites O_x; it is issued after this warp's next arrive on P_x
     }
   }
 
@@ -301,6 +415,41 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem, C::TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// planning kernel: one entry per (sequence, query tile), tiles with the longest key range first
+// ------------------------------------------------------------------------------------------------
+constexpr int PLAN_THREADS = 1024;
+constexpr int PLAN_MAX_LEVELS = 2048;   // query tiles per sequence the planner can order (256 K tokens)
+
+__global__ void __launch_bounds__(PLAN_THREADS) prefill_plan_kernel(const int32_t* cu_seqlens, int batch, int max_tiles,
+                                                                    int4* plan) {
+  // level t holds every sequence with more than t query tiles; levels are laid out from the highest down
+  __shared__ int cnt[PLAN_MAX_LEVELS];      // sequences per level, then the level's cursor
+  __shared__ int off[PLAN_MAX_LEVELS];      // first entry of the level
+  for (int t = threadIdx.x; t < max_tiles; t += PLAN_THREADS) cnt[t] = 0;
+  __syncthreads();
+  for (int b = threadIdx.x; b < batch; b += PLAN_THREADS) {
+    const int n = (cu_seqlens[b + 1] - cu_seqlens[b] + BM - 1) / BM;
+    if (n > 0) atomicAdd(&cnt[min(n, max_tiles) - 1], 1);   // histogram by tile count first
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int seqs = 0, entries = 0;
+    for (int t = max_tiles - 1; t >= 0; --t) {
+      seqs += cnt[t];          // sequences with more than t tiles
+      off[t] = entries;
+      entries += seqs;
+      cnt[t] = 0;
+    }
+  }
+  __syncthreads();
+  for (int b = threadIdx.x; b < batch; b += PLAN_THREADS) {
+    const int lo = cu_seqlens[b], len = cu_seqlens[b + 1] - lo;
+    const int n = min((len + BM - 1) / BM, max_tiles);
+    for (int t = 0; t < n; ++t) plan[off[t] + atomicAdd(&cnt[t], 1)] = make_int4(lo + t * BM, len - t * BM, t, b);
   }
 }
 
@@ -331,12 +480,24 @@ bool make_map(CUtensorMap* map, const void* ptr, int heads, int total) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+int sm_count() {
+  static std::atomic<int> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 1;
+  if (dev >= 0 && dev < 64 && cached[dev].load(std::memory_order_relaxed) > 0) return cached[dev].load(std::memory_order_relaxed);
+  int n = 0;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 1;
+  if (dev >= 0 && dev < 64) cached[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
+
 template <int NT>
-cudaError_t launch_nt(const PrefillArgs& a, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                      const TcParams& p, cudaStream_t st) {
+cudaError_t launch_nt(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, TcParams p, cudaStream_t st) {
   cudaError_t e = ensure_dynamic_smem<prefill_tc_kernel<NT>>(Cfg<NT>::SMEM_BYTES);
   if (e != cudaSuccess) return e;
-  dim3 grid((a.max_seqlen + BM - 1) / BM, a.Hq / NT, a.batch);
+  p.n_hp = p.Hq / NT;
+  p.n_items *= p.n_hp;
+  const int grid = p.n_items < sm_count() ? p.n_items : sm_count();
   prefill_tc_kernel<NT><<<grid, Cfg<NT>::THREADS, Cfg<NT>::SMEM_BYTES, st>>>(mq, mk, mv, p);
   note_launch();
   return cudaGetLastError();
@@ -344,21 +505,34 @@ cudaError_t launch_nt(const PrefillArgs& a, const CUtensorMap& mq, const CUtenso
 
 }  // namespace
 
-bool prefill_tc_supported(const PrefillArgs& a, int total_tokens) {
-  return a.dtype == EARN_BF16 && a.D == HD && total_tokens >= BM;
+int prefill_plan_entries(const earn_batch_t& b) {
+  int64_t n = 0;
+  for (int i = 0; i < b.batch; ++i) n += (b.cu_seqlens_host[i + 1] - b.cu_seqlens_host[i] + BM - 1) / BM;
+  return n > INT32_MAX ? INT32_MAX : (int)n;
 }
 
-cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int32_t* status_word, cudaStream_t st) {
+bool prefill_tc_supported(const PrefillArgs& a, int total_tokens) {
+  return a.dtype == EARN_BF16 && a.D == HD && total_tokens >= BM && (a.max_seqlen + BM - 1) / BM <= PLAN_MAX_LEVELS;
+}
+
+cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int plan_entries, void* plan, int32_t* status_word,
+                              cudaStream_t st) {
   CUtensorMap mq, mk, mv;
   if (!make_map(&mq, a.q, a.Hq, total_tokens) || !make_map(&mk, a.k, a.Hkv, total_tokens) ||
       !make_map(&mv, a.v, a.Hkv, total_tokens))
     return cudaErrorInvalidValue;
+  if (plan_entries <= 0) return cudaSuccess;
+  prefill_plan_kernel<<<1, PLAN_THREADS, 0, st>>>(a.cu_seqlens, a.batch, (a.max_seqlen + BM - 1) / BM,
+                                                  reinterpret_cast<int4*>(plan));
+  note_launch();
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
   TcParams p{};
-  p.o = a.o; p.lse = a.lse; p.cu_seqlens = a.cu_seqlens; p.status = status_word;
-  p.Hq = a.Hq; p.g = a.Hq / a.Hkv; p.total = total_tokens;
+  p.o = a.o; p.lse = a.lse; p.plan = reinterpret_cast<const int4*>(plan); p.status = status_word;
+  p.Hq = a.Hq; p.g = a.Hq / a.Hkv; p.total = total_tokens; p.n_items = plan_entries;
   p.scale_log2 = a.scale * kLog2e;
-  // two query heads of one kv head per CTA when the group size allows it
-  return (p.g % 2 == 0) ? launch_nt<2>(a, mq, mk, mv, p, st) : launch_nt<1>(a, mq, mk, mv, p, st);
+  // two query heads of one kv head per work item when the group size allows it
+  return (p.g % 2 == 0) ? launch_nt<2>(mq, mk, mv, p, st) : launch_nt<1>(mq, mk, mv, p, st);
 }
 
 }  // namespace earn
