@@ -95,6 +95,44 @@ __device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
       "mov.b64 {%0, %1}, rd;\n\t}"
       : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
 }
+__device__ __forceinline__ void add2s(float& d0, float& d1, float a0, float a1, float c) {   // d = a + c
+  asm("{\n\t.reg .b64 ra, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rc, {%4, %4};\n\tadd.rn.ftz.f32x2 rd, ra, rc;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(c));
+}
+__device__ __forceinline__ void sub2(float& d0, float& d1, float a0, float a1, float b0, float b1) {   // d = a - b
+  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tsub.rn.ftz.f32x2 rd, ra, rb;\n\t"
+      "mov.b64 {%0, %1}, rd;\n\t}"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ void fma2v(float& d0, float& d1, float b0, float b1, float c) {   // d = d * b + c
+  asm("{\n\t.reg .b64 rb, rc, rd;\n\tmov.b64 rd, {%0, %1};\n\tmov.b64 rb, {%2, %3};\n\tmov.b64 rc, {%4, %4};\n\t"
+      "fma.rn.ftz.f32x2 rd, rd, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+      : "+f"(d0), "+f"(d1) : "f"(b0), "f"(b1), "f"(c));
+}
+
+// 2^x for a pair of lanes on the FMA pipe instead of the special-function unit: x = n + f with n = round(x),
+// f in [-1/2, 1/2]; 2^f by a cubic (relative error 7.5e-5, far below the bf16 rounding of P); the integer n is
+// added into the exponent field.  x is clamped at -126, so a masked (-inf) logit gives 2^-126, which vanishes
+// against the row sum.  Used for a fixed share of the columns so that both pipes work at the same time.
+__device__ __forceinline__ void exp2_poly2(float& e0, float& e1, float x0, float x1) {
+  constexpr float MAGIC = 12582912.f;   // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+  x0 = fmaxf(x0, -126.f);
+  x1 = fmaxf(x1, -126.f);
+  float t0, t1, n0, n1, f0, f1, p0, p1;
+  add2s(t0, t1, x0, x1, MAGIC);
+  add2s(n0, n1, t0, t1, -MAGIC);
+  sub2(f0, f1, x0, x1, n0, n1);
+  fma2(p0, p1, f0, f1, 0.055171460f, 0.24261086f);
+  fma2v(p0, p1, f0, f1, 0.69326097f);
+  fma2v(p0, p1, f0, f1, 0.99992812f);
+  e0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
+  e1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
+}
+#ifndef EARN_POLY_MASK
+#define EARN_POLY_MASK 0x5252u   // which of the 16 column pairs of a 32-column chunk take the polynomial (6 of 16)
+#endif
+
 template <int NT>
 __global__ void __launch_bounds__(Cfg<NT>::THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -293,39 +331,90 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         tc_fence_after();
         const bool diag = j == it.n_tiles - 1;        // key column c of this tile is visible to row r iff c <= r
         const int n_chunks = diag ? wq + 1 : 4;       // 32-column chunks with a visible key for this warp's rows
-        uint32_t a[32], b[32];
-        // ---- pass 1: row maximum
-        float mx = -INFINITY;
-        tmem_ld_32x32(t_s, a);
-        tmem_wait_ld(a);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          if (q < n_chunks) {
-            uint32_t(&cur)[32] = (q & 1) ? b : a;
-            uint32_t(&nxt)[32] = (q & 1) ? a : b;
-            if (q + 1 < n_chunks) tmem_ld_32x32(t_s + (q + 1) * 32, nxt);
-            if (diag && q == wq) {
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (c > lane) cur[c] = 0xff800000u;   // -inf
-            }
-#pragma unroll
-            for (int c = 0; c < 32; c += 2) mx = max3(mx, __uint_as_float(cur[c]), __uint_as_float(cur[c + 1]));
-            if (q + 1 < n_chunks) tmem_wait_ld(nxt);
-          }
-        }
-        mx *= sl2;
-        float alpha = 1.f;
-        bool grow = false;
+        uint32_t a[32], b[32], pk[4][16];
         if (j == 0) {
-          m_ref = mx;
-        } else if (mx > m_ref + RESCALE_THRESHOLD) {
-          alpha = ex2(m_ref - mx);
-          m_ref = mx;
-          grow = true;
+          // ---- first tile of the item: the reference is its own row maximum, found in a pass of its own
+          float mx = -INFINITY;
+          tmem_ld_32x32(t_s, a);
+          if (n_chunks > 1) tmem_ld_32x32(t_s + 32, b);
+          tmem_wait_ld(a);
+          tmem_wait_ld(b);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            if (q < n_chunks) {
+              uint32_t(&cur)[32] = (q & 1) ? b : a;
+              if (diag && q == wq) {
+#pragma unroll
+                for (int c = 0; c < 32; ++c)
+                  if (c > lane) cur[c] = 0xff800000u;   // -inf
+              }
+              float m1 = -INFINITY;
+#pragma unroll
+              for (int c = 0; c < 32; c += 4) {
+                mx = max3(mx, __uint_as_float(cur[c]), __uint_as_float(cur[c + 1]));
+                m1 = max3(m1, __uint_as_float(cur[c + 2]), __uint_as_float(cur[c + 3]));
+              }
+              mx = fmaxf(mx, m1);
+            }
+            if (q == 1 && n_chunks > 2) {
+              tmem_ld_32x32(t_s + 64, a);
+              if (n_chunks > 3) tmem_ld_32x32(t_s + 96, b);
+              tmem_wait_ld(a);
+              tmem_wait_ld(b);
+            }
+          }
+          m_ref = mx * sl2;
         }
-        if (__any_sync(0xffffffffu, grow)) {
+        // ---- P = 2^(S * scale - m_ref) as bf16 pairs (kept in registers until the reference is known to hold),
+        //      row sum and row maximum in the same pass.  If the maximum outgrew the reference by more than the
+        //      threshold (rare: the reference already covers every earlier tile), raise it, rescale what has been
+        //      accumulated, and redo the pass; S_x is still intact because nothing has been written over it.
+        float ls0, ls1;
+#pragma unroll 1
+        for (int attempt = 0;; ++attempt) {
+          const float neg_m = -m_ref;
+          float mx = -INFINITY;
+          ls0 = ls1 = 0.f;
+          tmem_ld_32x32(t_s, a);
+          tmem_wait_ld(a);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            if (q < n_chunks) {
+              uint32_t(&cur)[32] = (q & 1) ? b : a;
+              uint32_t(&nxt)[32] = (q & 1) ? a : b;
+              if (q + 1 < n_chunks) tmem_ld_32x32(t_s + (q + 1) * 32, nxt);
+              if (diag && q == wq) {
+#pragma unroll
+                for (int c = 0; c < 32; ++c)
+                  if (c > lane) cur[c] = 0xff800000u;
+              }
+#pragma unroll
+              for (int c = 0; c < 32; c += 2) {
+                const float s0 = __uint_as_float(cur[c]), s1 = __uint_as_float(cur[c + 1]);
+                mx = max3(mx, s0, s1);
+                float e0, e1;
+                fma2(e0, e1, s0, s1, sl2, neg_m);
+                if ((EARN_POLY_MASK >> (c >> 1)) & 1u) {
+                  exp2_poly2(e0, e1, e0, e1);
+                } else {
+                  e0 = ex2(e0);
+                  e1 = ex2(e1);
+                }
+                add2(ls0, ls1, e0, e1);
+                pk[q][c >> 1] = pack_bf16(e0, e1);
+              }
+              if (q + 1 < n_chunks) tmem_wait_ld(nxt);
+            } else {
+#pragma unroll
+              for (int c = 0; c < 16; ++c) pk[q][c] = 0u;
+            }
+          }
+          const float mxs = mx * sl2;
+          const bool grow = mxs > m_ref + RESCALE_THRESHOLD;
+          if (attempt > 0 || !__any_sync(0xffffffffu, grow)) break;
           // S_x(j) was issued after P_x V of tile j-1, so the commit that signalled it covers that too: O_x is quiescent
+          const float alpha = grow ? ex2(m_ref - mxs) : 1.f;
+          if (grow) m_ref = mxs;
           l0 *= alpha;
           l1 *= alpha;
 #pragma unroll
@@ -337,39 +426,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             tmem_st_32x32(t_o + q * 32, a);
           }
         }
-        // ---- pass 2: P = 2^(S * scale - m_ref) as bf16 pairs, written over the consumed columns of S_x
-        const float neg_m = -m_ref;
-        tmem_ld_32x32(t_s, a);
-        tmem_wait_ld(a);
+        l0 += ls0;
+        l1 += ls1;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          uint32_t pk[16];
-          if (q < n_chunks) {
-            uint32_t(&cur)[32] = (q & 1) ? b : a;
-            uint32_t(&nxt)[32] = (q & 1) ? a : b;
-            if (q + 1 < n_chunks) tmem_ld_32x32(t_s + (q + 1) * 32, nxt);
-            if (diag && q == wq) {
-#pragma unroll
-              for (int c = 0; c < 32; ++c)
-                if (c > lane) cur[c] = 0xff800000u;
-            }
-#pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-              float e0, e1;
-              fma2(e0, e1, __uint_as_float(cur[c]), __uint_as_float(cur[c + 1]), sl2, neg_m);
-              e0 = ex2(e0);
-              e1 = ex2(e1);
-              add2(l0, l1, e0, e1);
-              pk[c >> 1] = pack_bf16(e0, e1);
-            }
-            tmem_st_32x16(t_s + q * 16, pk);
-            if (q + 1 < n_chunks) tmem_wait_ld(nxt);
-          } else {
-#pragma unroll
-            for (int c = 0; c < 16; ++c) pk[c] = 0u;
-            tmem_st_32x16(t_s + q * 16, pk);
-          }
-        }
+        for (int q = 0; q < 4; ++q) tmem_st_32x16(t_s + q * 16, pk[q]);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar(C::BAR_P + x));
