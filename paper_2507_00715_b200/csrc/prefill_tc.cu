@@ -229,33 +229,42 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp runs the loop (so that every descriptor is warp-uniform arithmetic and nothing but the
+    // tcgen05.mma instructions themselves sits between two of them); lane 0 issues.
+    {
+      const bool leader = lane == 0;
       constexpr uint32_t idesc_s = idesc_bf16_f32(BM, BN, 0, 0);   // Q (K-major) x K^T (K-major)
       constexpr uint32_t idesc_o = idesc_bf16_f32(BM, HD, 0, 1);   // P (TMEM) x V (MN-major)
-      auto wait_full = [&](int e) {
-        return mbar_wait_bounded(bar(C::BAR_FULL + e % C::NSTAGE), (e / C::NSTAGE) & 1, abort_flag, WAIT_LIMIT);
+      constexpr uint32_t desc_hi = smem_desc_hi_sw128(1024);
+      const uint32_t q_lo = smem_desc_lo(sQ, 16), k_lo = smem_desc_lo(sRing, 16), v_lo = smem_desc_lo(sRing, HALF);
+      auto wait = [&](int b, int parity) {   // warp-uniform result
+        return __all_sync(0xffffffffu, mbar_wait_bounded(bar(b), (uint32_t)parity & 1u, abort_flag, WAIT_LIMIT));
       };
+      auto wait_full = [&](int e) { return wait(C::BAR_FULL + e % C::NSTAGE, e / C::NSTAGE); };
       // S_x = Q_x K^T with the K tile of ring entry e; `last` = no later S of this item reads Q_x
       auto issue_s = [&](int x, int e, bool last) {
-        const uint32_t sK = sRing + (e % C::NSTAGE) * TILE;
+        const uint32_t a0 = q_lo + x * (TILE >> 4), b0 = k_lo + (e % C::NSTAGE) * (TILE >> 4);
+        if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < HD / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * HALF + (kk & 3) * 32;
-          umma_ss(tmem + x * 128, smem_desc_sw128(sQ + x * TILE + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024),
-                  idesc_s, kk > 0);
+          for (int kk = 0; kk < HD / 16; ++kk) {
+            const uint32_t off = ((kk >> 2) * HALF + (kk & 3) * 32) >> 4;
+            umma_ss_lohi(tmem + x * 128, a0 + off, desc_hi, b0 + off, desc_hi, idesc_s, kk > 0);
+          }
+          umma_commit(bar(C::BAR_S + x));
+          if (last) umma_commit(bar(C::BAR_QFREE + x));
+          if (x == NT - 1) umma_commit(bar(C::BAR_EMPTY + e % C::NSTAGE));   // K tile free once the last S has read it
         }
-        umma_commit(bar(C::BAR_S + x));
-        if (last) umma_commit(bar(C::BAR_QFREE + x));
-        if (x == NT - 1) umma_commit(bar(C::BAR_EMPTY + e % C::NSTAGE));   // K tile free once the last S has read it
       };
       // O_x (+)= P_x V with P_x in tensor memory (bf16 pairs over the first 64 columns of S_x) and the V tile of entry e
       auto issue_pv = [&](int x, int e, bool first_tile) {
-        const uint32_t sV = sRing + (e % C::NSTAGE) * TILE;
+        const uint32_t b0 = v_lo + (e % C::NSTAGE) * (TILE >> 4);
+        if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < BN / 16; ++kk)
-          umma_ts(tmem + (NT + x) * 128, tmem + x * 128 + kk * 8, smem_desc_sw128(sV + kk * 2048, HALF, 1024), idesc_o,
-                  (!first_tile || kk > 0) ? 1u : 0u);
-        if (x == NT - 1) umma_commit(bar(C::BAR_EMPTY + e % C::NSTAGE));   // V tile free once the last P V has read it
+          for (int kk = 0; kk < BN / 16; ++kk)
+            umma_ts_lohi(tmem + (NT + x) * 128, tmem + x * 128 + kk * 8, b0 + kk * (2048 >> 4), desc_hi, idesc_o,
+                         (!first_tile || kk > 0) ? 1u : 0u);
+          if (x == NT - 1) umma_commit(bar(C::BAR_EMPTY + e % C::NSTAGE));   // V tile free once the last P V has read it
+        }
       };
       int eb = 0;       // ring entry of the current item's K_0
       int n_item = 0;   // items started so far
@@ -266,7 +275,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       if (ok) {
         cur = load_item(p, first, NT);
         for (int x = 0; x < NT && ok; ++x) {
-          ok = mbar_wait_bounded(bar(C::BAR_QFULL + x), 0, abort_flag, WAIT_LIMIT) && (x > 0 || wait_full(0));
+          ok = wait(C::BAR_QFULL + x, 0) && (x > 0 || wait_full(0));
           if (!ok) break;
           tc_fence_after();
           issue_s(x, 0, cur.n_tiles == 1);
@@ -279,7 +288,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int n = cur.n_tiles;
         for (int j = 0; j < n && ok; ++j) {
           for (int x = 0; x < NT && ok; ++x) {
-            ok = mbar_wait_bounded(bar(C::BAR_P + x), n_p[x] & 1, abort_flag, WAIT_LIMIT);   // P_x(j) written, S_x consumed
+            ok = wait(C::BAR_P + x, n_p[x]);   // P_x(j) written, S_x consumed
             ++n_p[x];
             if (ok && x == 0) ok = wait_full(eb + 2 * j + 1);
             if (!ok) break;
@@ -291,9 +300,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
               tc_fence_after();
               issue_s(x, eb + 2 * j + 2, j + 1 == n - 1);
             } else {
-              umma_commit(bar(C::BAR_O + x));
+              if (leader) umma_commit(bar(C::BAR_O + x));
               if (has_next) {   // straight on to the next item: its Q_x and first K tile are on their way already
-                ok = mbar_wait_bounded(bar(C::BAR_QFULL + x), (n_item + 1) & 1, abort_flag, WAIT_LIMIT);
+                ok = wait(C::BAR_QFULL + x, n_item + 1);
                 if (ok && x == 0) ok = wait_full(eb + 2 * n);
                 if (!ok) break;
                 tc_fence_after();
@@ -305,11 +314,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         eb += 2 * n;
         cur = nxt;
       }
-      if (*abort_flag) {
+      if (leader && *abort_flag) {
         int none = 0;
         umma_commit(bar(C::BAR_DRAIN));   // everything this thread issued has retired once this fires
         mbar_wait_bounded(bar(C::BAR_DRAIN), 0, &none, WAIT_LIMIT);
       }
+      __syncwarp();
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ softmax warpgroup x, one row per thread
