@@ -217,9 +217,11 @@ class DecodeState:
         self.priv_k: List[List[np.ndarray]] = [[] for _ in range(n)]
         self.priv_v: List[List[np.ndarray]] = [[] for _ in range(n)]
 
-    def step(self, q, k_new, v_new, parents: Optional[Sequence[int]] = None) -> np.ndarray:
+    def step(self, q, k_new, v_new, parents: Optional[Sequence[int]] = None, rows=None) -> np.ndarray:
         """q [B*W,Hq,D], k_new,v_new [B*W,Hkv,D]; parents[j] in [0,W) = the beam of the same
-        sequence whose generated history beam j continues.  Returns O float64 [B*W,Hq,D]."""
+        sequence whose generated history beam j continues.  Returns O float64 [B*W,Hq,D].
+        rows: optional set of (beam, query head) pairs; the cache is updated for every beam but only
+        those outputs are computed (the others stay zero) -- for workloads too large to compute in full."""
         w = self.beams
         n = len(self.priv_k)
         if parents is not None:
@@ -235,9 +237,13 @@ class DecodeState:
             self.priv_k[j].append(np.asarray(k_new[j], dtype=np.float64))   # Eq. 4: append first,
             self.priv_v[j].append(np.asarray(v_new[j], dtype=np.float64))   # then attend (self included)
             b = j // w
+            if rows is not None and not any((j, h) in rows for h in range(hq)):
+                continue
             gen_k = np.stack(self.priv_k[j], axis=0)
             gen_v = np.stack(self.priv_v[j], axis=0)
             for h in range(hq):
+                if rows is not None and (j, h) not in rows:
+                    continue
                 keys = np.concatenate([self.shared_k[b][:, h // g, :], gen_k[:, h // g, :]], axis=0)
                 vals = np.concatenate([self.shared_v[b][:, h // g, :], gen_v[:, h // g, :]], axis=0)
                 out[j, h] = decode_attention(q[j, h], keys, vals, self.scale)

@@ -60,3 +60,49 @@ def test_group_of_three_and_odd_register_count():
     # g*R = 3*7 = 21 rows: a ragged last row tile that straddles two heads
     run_workload_and_compare(BASE.replace(seed=21, n_q_heads=6, n_kv_heads=2, r_head=3, r_tail=4, lens=(60, 33), batch=2,
                                           beams=2, decode_steps=4))
+
+
+def test_register_layers_ignore_prompt_tokens_on_the_gpu():
+    """Overwriting every non-register K/V/Q row of a register layer changes nothing, bit for bit: compact cache,
+    register attention and every decode output of that layer (the layer never reads those rows)."""
+    from parity_util import make_session
+    from oracle import earn_oracle as orc
+
+    w = BASE.replace(seed=22, lens=(300, 129, 64), r_head=6, r_tail=5, decode_steps=3, beams=2, n_layers=2, split_k=1)
+    idx = orc.register_indices(wl.seqlens(w), w.r_head, w.r_tail)
+    cu = wl.cu_seqlens(w)
+    keep = torch.zeros(int(cu[-1]), dtype=torch.bool)
+    for b in range(w.batch):
+        keep[cu[b] + torch.from_numpy(idx[b]).long()] = True
+    outs = []
+    for noise_seed in (None, 1234):
+        ses = make_session(w)
+        q, k, v = wl.layer_qkv(w, 1, "cuda")
+        if noise_seed is not None:
+            g = torch.Generator(device="cuda").manual_seed(noise_seed)
+            for t in (q, k, v):
+                noise = torch.randn(t.shape, generator=g, device="cuda").to(t.dtype)
+                t[~keep.cuda()] = noise[~keep.cuda()]
+        got = [ses.prefill_layer(1, q, k, v).clone(), ses.k_shared[1].clone(), ses.v_shared[1].clone()]
+        for step in range(1, w.decode_steps + 1):
+            parents = wl.beam_parents(w, step) if step > 1 else None
+            ses.begin_step(step, None if parents is None else torch.from_numpy(parents).cuda())
+            got.append(ses.decode_layer(1, step, *wl.decode_qkv(w, 1, step, "cuda")).clone())
+        outs.append(got)
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
+def test_batch_order_does_not_matter():
+    """Sequences are independent (varlen packing, no padding): reversing the batch reverses the outputs."""
+    from parity_util import make_session
+
+    w = BASE.replace(seed=23, lens=(200, 77, 333), n_layers=1, split_k=1, decode_steps=0)
+    cu = wl.cu_seqlens(w)
+    q, k, v = wl.layer_qkv(w, 0, "cuda")
+    o = make_session(w).prefill_layer(0, q, k, v)
+    order = [2, 1, 0]
+    pieces = lambda t: torch.cat([t[cu[b]:cu[b + 1]] for b in order])   # noqa: E731
+    w2 = w.replace(lens=tuple(w.lens[b] for b in order))
+    o2 = make_session(w2).prefill_layer(0, pieces(q), pieces(k), pieces(v))
+    assert torch.equal(o2, pieces(o))
