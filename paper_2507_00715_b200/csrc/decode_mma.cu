@@ -4,7 +4,8 @@
 // loads in flight with few instructions, not around the tensor cores; warp-level mma.sync (m16n8k16)
 // only keeps the few query rows per key (g heads x W beams, padded to 16) off the FMA pipe.
 //
-// One CTA = (sequence b, kv head, split of the shared segment, tile of 16 query rows); 1 warp.  The key
+// One CTA = (sequence b, kv head, split of the shared segment, tile of 16 query rows); one warp, or four
+// warps that deal the tiles of a short list among themselves when the grid is small.  The key
 // list of a CTA is its chunk of the shared segment (the prompt K/V of a layer l < k read in place, or
 // the compact register pages of a layer l >= k) followed -- in split 0 only -- by the generated tokens
 // of the beams its rows belong to (masked per row to the row's own beam; the newest token comes
@@ -33,17 +34,13 @@ using namespace mma;
 #ifndef EARN_DECODE_KT
 #define EARN_DECODE_KT 16
 #endif
-#ifndef EARN_DECODE_NWARPS
-#define EARN_DECODE_NWARPS 1
-#endif
 #ifndef EARN_DECODE_STAGES
 #define EARN_DECODE_STAGES 4
 #endif
 constexpr int KT = EARN_DECODE_KT;           // list positions per tile (16 or 32)
-constexpr int NWARPS = EARN_DECODE_NWARPS;   // warps per CTA; tiles are dealt round-robin to them
 constexpr int N8 = KT / 8, H16 = KT / 16;
 
-template <int D, int STAGES>   // STAGES: cp.async ring depth per warp
+template <int D, int STAGES, int NWARPS>   // STAGES: cp.async ring depth per warp; NWARPS: warps per CTA, tiles dealt round-robin
 struct Geo {
   static constexpr int ROWB = D * 2;            // bytes of one K (or V) row
   static constexpr int PITCH = ROWB + 16;       // padded row pitch: conflict-free ldmatrix, 16-byte aligned
@@ -55,10 +52,10 @@ struct Geo {
   static constexpr int SMEM_B = DATA_B;
 };
 
-template <int D, int STAGES>
+template <int D, int STAGES, int NWARPS>
 __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   using bf16 = __nv_bfloat16;
-  using G = Geo<D, STAGES>;
+  using G = Geo<D, STAGES, NWARPS>;
   constexpr int KSTEPS = D / 16, NTILES = D / 8;
   extern __shared__ __align__(128) uint8_t smem[];
 
@@ -285,6 +282,29 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
   __syncthreads();   // all rings are idle: reuse the shared memory for the merge
 
+  if (NWARPS == 1 && a.plan.n_splits <= 1) {
+    // one warp saw the whole key list: normalise, stage the 16 x D bf16 tile, 16-byte stores
+    const float i0 = 1.f / l0, i1 = 1.f / l1;   // rows past W*g hold garbage and are not stored
+    const int r0 = lane >> 2, r1 = r0 + 8;
+#pragma unroll
+    for (int n = 0; n < NTILES; ++n) {
+      *reinterpret_cast<uint32_t*>(smem + r0 * G::PITCH + (n * 8 + c2) * 2) = pack2(o[n][0] * i0, o[n][1] * i0);
+      *reinterpret_cast<uint32_t*>(smem + r1 * G::PITCH + (n * 8 + c2) * 2) = pack2(o[n][2] * i1, o[n][3] * i1);
+    }
+    const int rr = row0 + (lane & 15);   // lane r (and r + 16) resolves output row r; the store loop fetches it by shuffle
+    const int64_t my_off = rr < n_rows ? (((int64_t)b * W + rr / g) * a.Hq + kvh * g + rr % g) * D : -1;
+    __syncwarp();
+    bf16* og = reinterpret_cast<bf16*>(a.o);
+#pragma unroll
+    for (int it = 0; it < 16 / RPI; ++it) {
+      const int r = it * RPI + lane / CH, chunk = lane % CH;
+      const int64_t off = __shfl_sync(0xffffffffu, my_off, r);
+      if (off >= 0)
+        *reinterpret_cast<uint4*>(og + off + chunk * 8) = *reinterpret_cast<const uint4*>(smem + r * G::PITCH + chunk * 16);
+    }
+    return;
+  }
+
   float* mo = reinterpret_cast<float*>(smem);                 // [NWARPS][16][D]
   float* ml = mo + NWARPS * 16 * D;                           // [NWARPS][16][2] = (m, l)
   {
@@ -392,14 +412,14 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   }
 }
 
-template <int D, int ST>
+template <int D, int ST, int NWARPS>
 cudaError_t launch_d(const DecodeArgs& a, cudaStream_t st) {
-  constexpr int smem = Geo<D, ST>::SMEM_B;
-  cudaError_t e = ensure_dynamic_smem<decode_mma_kernel<D, ST>>(smem);
+  constexpr int smem = Geo<D, ST, NWARPS>::SMEM_B;
+  cudaError_t e = ensure_dynamic_smem<decode_mma_kernel<D, ST, NWARPS>>(smem);
   if (e != cudaSuccess) return e;
   const int splits = a.plan.n_splits > 0 ? a.plan.n_splits : 1;
   dim3 grid(splits * a.plan.row_tiles, a.Hkv, a.batch);
-  decode_mma_kernel<D, ST><<<grid, NWARPS * 32, smem, st>>>(a);
+  decode_mma_kernel<D, ST, NWARPS><<<grid, NWARPS * 32, smem, st>>>(a);
   note_launch();
   return cudaGetLastError();
 }
@@ -407,12 +427,20 @@ cudaError_t launch_d(const DecodeArgs& a, cudaStream_t st) {
 }  // namespace
 
 cudaError_t launch_decode_mma(const DecodeArgs& a, int max_shared_len, cudaStream_t st) {
-  // a key list of at most two tiles needs no deep ring: a small footprint keeps every CTA resident at once
+  // One warp per CTA with a deep ring streams best whenever the grid covers the GPU (measured on B200 at the 7B
+  // shapes: 8.9 us per compact-cache layer against 13.0 us with four warps).  A short key list on a grid of less
+  // than a CTA per SM is latency-bound instead: four warps take a tile or two each (5.9 against 6.8 us at the 1.5B
+  // shapes).  A list of at most two tiles needs no deep ring either way.
   const int g = a.Hq / a.Hkv;
   const int beams_per_tile = a.beams < (16 + g - 1) / g + 1 ? a.beams : (16 + g - 1) / g + 1;
-  const bool small = a.plan.n_splits <= 1 && max_shared_len + beams_per_tile * a.step <= 2 * KT * NWARPS;
-  if (a.D == 64) return small ? launch_d<64, 2>(a, st) : launch_d<64, EARN_DECODE_STAGES>(a, st);
-  return small ? launch_d<128, 2>(a, st) : launch_d<128, EARN_DECODE_STAGES>(a, st);
+  const int max_tiles = (max_shared_len + beams_per_tile * a.step + KT - 1) / KT;
+  const long ctas = (long)(a.plan.n_splits > 0 ? a.plan.n_splits : 1) * a.plan.row_tiles * a.Hkv * a.batch;
+  const bool unsplit = a.plan.n_splits <= 1;
+  const bool four_warps = unsplit && max_tiles <= 16 && ctas < 148;
+  const bool small = unsplit && max_tiles <= 2;
+  if (a.D == 64)
+    return four_warps ? launch_d<64, 2, 4>(a, st) : small ? launch_d<64, 2, 1>(a, st) : launch_d<64, EARN_DECODE_STAGES, 1>(a, st);
+  return four_warps ? launch_d<128, 2, 4>(a, st) : small ? launch_d<128, 2, 1>(a, st) : launch_d<128, EARN_DECODE_STAGES, 1>(a, st);
 }
 
 }  // namespace earn

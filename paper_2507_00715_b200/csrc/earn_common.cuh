@@ -55,7 +55,8 @@ size_t workspace_head_bytes(const earn_model_t& m, const earn_batch_t& b, int be
 
 void note_launch(int n = 1);   // host-side count of kernels launched by this library
 
-// Opt a kernel in to `bytes` of dynamic shared memory, once per device (the attribute call is not free).
+// Opt a kernel in to `bytes` of dynamic shared memory and the largest carveout, once per device (the attribute
+// calls are not free).
 template <auto Kernel>
 cudaError_t ensure_dynamic_smem(int bytes) {
   static std::atomic<uint64_t> done{0};   // one bit per device ordinal < 64
@@ -64,6 +65,9 @@ cudaError_t ensure_dynamic_smem(int bytes) {
   if (e != cudaSuccess) return e;
   if (dev < 64 && ((done.load(std::memory_order_relaxed) >> dev) & 1)) return cudaSuccess;
   e = cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  // ask for the largest shared-memory carveout: left to itself the driver may size it for a single CTA
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(Kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
   if (e == cudaSuccess && dev < 64) done.fetch_or(1ull << dev, std::memory_order_relaxed);
   return e;
 }

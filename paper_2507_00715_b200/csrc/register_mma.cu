@@ -4,10 +4,11 @@
 // The work per sequence is tiny (R <= 128 keys), so the kernel is shaped for HBM traffic and latency:
 // one CTA per (sequence, kv head) brings that head's compact K and V rows into shared memory once
 // (through the page table) and all g query heads of the group use them.  The g*R query rows
-// (row = head-in-group * R + register index) are cut into tiles of 16; each of the 8 warps takes
-// tiles round-robin, keeps its Q fragments in registers, runs mma.sync m16n8k16 over 16-key tiles up
-// to the causal limit with an online softmax in the log2 domain, and writes its 16 output rows
-// through a private shared-memory staging tile as 16-byte stores.
+// (row = head-in-group * R + register index) are cut into tiles of 16; each of the warps takes
+// tiles round-robin, copies its 16 query rows into a private shared-memory tile with 16-byte
+// asynchronous copies (in flight together with the K/V copies), reads them back as ldmatrix
+// fragments, runs mma.sync m16n8k16 over 16-key tiles up to the causal limit with an online softmax
+// in the log2 domain, and writes its 16 output rows through the same private tile as 16-byte stores.
 #include "earn_common.cuh"
 #include "mma_sync.cuh"
 #include "sm100_ptx.cuh"
@@ -16,7 +17,10 @@ namespace earn {
 namespace {
 using namespace mma;
 
-constexpr int NW = 8;
+#ifndef EARN_REGISTER_NW
+#define EARN_REGISTER_NW 4
+#endif
+constexpr int NW = EARN_REGISTER_NW;   // warps per CTA: few, so that several CTAs share an SM and one's loads overlap another's math
 constexpr int MAX_R = 128;
 
 template <int D>
@@ -26,7 +30,7 @@ struct RGeo {
 };
 
 template <int D>
-__global__ void __launch_bounds__(NW * 32) register_mma_kernel(RegisterArgs a, int r_pad) {
+__global__ void __launch_bounds__(NW * 32, 12 / NW) register_mma_kernel(RegisterArgs a, int r_pad) {
   using bf16 = __nv_bfloat16;
   using G = RGeo<D>;
   constexpr int KSTEPS = D / 16, NTILES = D / 8, CH = G::ROWB / 16;
@@ -35,7 +39,30 @@ __global__ void __launch_bounds__(NW * 32) register_mma_kernel(RegisterArgs a, i
   const int kvh = blockIdx.x, b = blockIdx.y;
   const int R = a.R, g = a.Hq / a.Hkv, n_rows = g * R;
   const uint32_t sK = ptx::smem_u32(smem), sV = sK + r_pad * G::PITCH;
-  uint8_t* gO = smem + 2 * r_pad * G::PITCH + warp * 16 * G::PITCH;
+  uint8_t* gO = smem + 2 * r_pad * G::PITCH + warp * 16 * G::PITCH;   // this warp's tile: Q rows in, O rows out
+  const uint32_t sQ = ptx::smem_u32(gO);
+  const bf16* qg = reinterpret_cast<const bf16*>(a.q_reg);
+  // Row r of a tile is query row (head in group, register index) = (rr / R, rr % R), rr = 16 * tile + r, and sits
+  // at the same element offset in q_reg and o_reg.  Lane r (and r + 16) works the offset out once per tile; the
+  // copy loops fetch it by shuffle (-1: the row does not exist).
+  constexpr int RPI = 32 / CH;   // rows covered by one 16-byte access of the whole warp
+  auto row_offset = [&](int tile) -> int64_t {
+    const int rr = tile * 16 + (lane & 15);
+    if (rr >= n_rows) return -1;
+    const int gi = rr / R, m = rr - gi * R;
+    return (((int64_t)b * R + m) * a.Hq + kvh * g + gi) * D;
+  };
+  // 16 query rows of a tile -> the warp's tile (rows past g*R become zero)
+  auto load_q_tile = [&](int64_t my_off) {
+#pragma unroll
+    for (int it = 0; it < 16 / RPI; ++it) {
+      const int r = it * RPI + lane / CH, ch = lane % CH;
+      const int64_t off = __shfl_sync(0xffffffffu, my_off, r);
+      cp_async16(sQ + r * G::PITCH + ch * 16, qg + (off < 0 ? 0 : off) + ch * 8, off < 0 ? 0 : 16);
+    }
+  };
+  int64_t tile_off = row_offset(warp);
+  if (warp * 16 < n_rows) load_q_tile(tile_off);
 
   // ---- compact K/V rows of this (sequence, kv head) -> shared memory; rows R..r_pad-1 are zero
   {
@@ -56,7 +83,6 @@ __global__ void __launch_bounds__(NW * 32) register_mma_kernel(RegisterArgs a, i
   const int mat = lane >> 3;
   const uint32_t k_lane = (uint32_t)(((mat >> 1) << 3) + (lane & 7)) * G::PITCH + (uint32_t)(mat & 1) * 16;
   const uint32_t v_lane = (uint32_t)(((mat & 1) << 3) + (lane & 7)) * G::PITCH + (uint32_t)(mat >> 1) * 16;
-  const bf16* qg = reinterpret_cast<const bf16*>(a.q_reg);
   bf16* og = reinterpret_cast<bf16*>(a.o_reg);
   cp_async_wait<0>();
   __syncthreads();   // every warp's copies have landed (warps without a tile take part too)
@@ -66,18 +92,17 @@ __global__ void __launch_bounds__(NW * 32) register_mma_kernel(RegisterArgs a, i
     // row -> (head in group, register index); rows past g*R read nothing and write nothing
     const int gi0 = rr0 / R, m0r = rr0 % R, gi1 = rr1 / R, m1r = rr1 % R;
     const bool ok0 = rr0 < n_rows, ok1 = rr1 < n_rows;
-    uint32_t qf[KSTEPS][4];
-    {
-      const bf16* q0 = qg + (((int64_t)b * R + m0r) * a.Hq + kvh * g + gi0) * D;
-      const bf16* q1 = qg + (((int64_t)b * R + m1r) * a.Hq + kvh * g + gi1) * D;
-#pragma unroll
-      for (int kk = 0; kk < KSTEPS; ++kk) {
-        qf[kk][0] = ok0 ? *reinterpret_cast<const uint32_t*>(q0 + kk * 16 + c2) : 0u;
-        qf[kk][1] = ok1 ? *reinterpret_cast<const uint32_t*>(q1 + kk * 16 + c2) : 0u;
-        qf[kk][2] = ok0 ? *reinterpret_cast<const uint32_t*>(q0 + kk * 16 + 8 + c2) : 0u;
-        qf[kk][3] = ok1 ? *reinterpret_cast<const uint32_t*>(q1 + kk * 16 + 8 + c2) : 0u;
-      }
+    if (tile != warp) {   // later tiles of this warp: the first one came in with the K/V rows
+      tile_off = row_offset(tile);
+      load_q_tile(tile_off);
+      cp_async_commit();
+      cp_async_wait<0>();
+      __syncwarp();
     }
+    uint32_t qf[KSTEPS][4];
+#pragma unroll
+    for (int kk = 0; kk < KSTEPS; ++kk)
+      ldsm_x4(sQ + (lane & 15) * G::PITCH + (lane >> 4) * 16 + kk * 32, qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3]);
     // causal limit of the tile: the largest register index among its rows
     const int first = tile * 16, last = min(first + 15, n_rows - 1);
     const int m_hi = (first / R == last / R) ? last % R : R - 1;
@@ -153,13 +178,16 @@ __global__ void __launch_bounds__(NW * 32) register_mma_kernel(RegisterArgs a, i
       }
     }
     __syncwarp();
-    for (int i = lane; i < 16 * CH; i += 32) {
-      const int r = i / CH, ch = i % CH, rr = tile * 16 + r;
-      if (rr < n_rows) {
+#pragma unroll
+    for (int it = 0; it < 16 / RPI; ++it) {
+      const int r = it * RPI + lane / CH, ch = lane % CH;
+      const int64_t off = __shfl_sync(0xffffffffu, tile_off, r);
+      if (off >= 0) {
         const uint4 v = *reinterpret_cast<const uint4*>(gO + r * G::PITCH + ch * 16);
-        *reinterpret_cast<uint4*>(og + (((int64_t)b * R + rr % R) * a.Hq + kvh * g + rr / R) * D + ch * 8) = v;
+        *reinterpret_cast<uint4*>(og + off + ch * 8) = v;
       }
     }
+    __syncwarp();   // the tile is free for the next Q rows
   }
 }
 
