@@ -10,6 +10,8 @@ namespace earn {
 namespace {
 
 __global__ void __launch_bounds__(128) compact_kernel(CompactArgs a) {
+  pdl_launch_dependents();
+  pdl_wait();   // everything below reads or writes global memory
   const int m = blockIdx.x, b = blockIdx.y;
   const int R = a.r_head + a.r_tail;
   const int lo = a.cu_seqlens[b], len = a.cu_seqlens[b + 1] - lo;
@@ -55,9 +57,9 @@ __global__ void beam_reparent_kernel(int beams, int max_new, int step, const int
 
 cudaError_t launch_compact(const CompactArgs& a, cudaStream_t st) {
   dim3 grid(a.r_head + a.r_tail, a.batch);
-  compact_kernel<<<grid, 128, 0, st>>>(a);
+  cudaError_t e = launch_pdl(compact_kernel, grid, dim3(128), 0, st, a);
   note_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_beam_reparent(int batch, int beams, int max_new, int step, const int32_t* parent,

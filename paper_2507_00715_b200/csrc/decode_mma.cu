@@ -58,6 +58,7 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   using G = Geo<D, STAGES, NWARPS>;
   constexpr int KSTEPS = D / 16, NTILES = D / 8;
   extern __shared__ __align__(128) uint8_t smem[];
+  pdl_wait();   // everything below reads or writes global memory
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.z, kvh = blockIdx.y;
@@ -276,6 +277,10 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
     __syncwarp();   // every lane is done with this stage before the next iteration refills it
   }
   cp_async_wait<0>();
+  // The next kernel on the stream may be scheduled from here on (once every CTA of this grid is past its key
+  // loop): releasing it earlier let its CTAs pile up on whichever SMs had room and unbalanced the next launch
+  // (55 us against 50 us per prompt-cache layer at the 7B shapes).
+  pdl_launch_dependents();
   l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
   l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
   l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
@@ -419,9 +424,9 @@ cudaError_t launch_d(const DecodeArgs& a, cudaStream_t st) {
   if (e != cudaSuccess) return e;
   const int splits = a.plan.n_splits > 0 ? a.plan.n_splits : 1;
   dim3 grid(splits * a.plan.row_tiles, a.Hkv, a.batch);
-  decode_mma_kernel<D, ST, NWARPS><<<grid, NWARPS * 32, smem, st>>>(a);
+  e = launch_pdl(decode_mma_kernel<D, ST, NWARPS>, grid, dim3(NWARPS * 32), smem, st, a);
   note_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace

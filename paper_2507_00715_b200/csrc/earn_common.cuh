@@ -72,6 +72,28 @@ cudaError_t ensure_dynamic_smem(int bytes) {
   return e;
 }
 
+// ---- programmatic dependent launch: a kernel launched through launch_pdl may start (be scheduled, set up its
+// shared memory and barriers) while the kernel before it on the stream is still running; it must call pdl_wait()
+// before it touches global memory, which returns once that kernel has completed and its writes are visible.
+// pdl_launch_dependents() lets the kernel after this one do the same.  Both are no-ops in an ordinary launch.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- launchers (one per .cu file); all return cudaGetLastError() of their launches ----
 struct PrefillArgs {
   const void *q, *k, *v;

@@ -176,6 +176,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const int first = blockIdx.x, stride = gridDim.x;   // this CTA's items: first, first + stride, ...
+  pdl_launch_dependents();
+  pdl_wait();   // the plan (written by the kernel launched just before this one) and every tensor are read below
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer: K/V ring
@@ -499,6 +501,8 @@ __global__ void __launch_bounds__(PLAN_THREADS) prefill_plan_kernel(const int32_
   // level t holds every sequence with more than t query tiles; levels are laid out from the highest down
   __shared__ int cnt[PLAN_MAX_LEVELS];      // sequences per level, then the level's cursor
   __shared__ int off[PLAN_MAX_LEVELS];      // first entry of the level
+  pdl_launch_dependents();
+  pdl_wait();   // the plan area may still be read by the kernel before this one
   for (int t = threadIdx.x; t < max_tiles; t += PLAN_THREADS) cnt[t] = 0;
   __syncthreads();
   for (int b = threadIdx.x; b < batch; b += PLAN_THREADS) {
@@ -568,9 +572,9 @@ cudaError_t launch_nt(const CUtensorMap& mq, const CUtensorMap& mk, const CUtens
   p.n_hp = p.Hq / NT;
   p.n_items *= p.n_hp;
   const int grid = p.n_items < sm_count() ? p.n_items : sm_count();
-  prefill_tc_kernel<NT><<<grid, Cfg<NT>::THREADS, Cfg<NT>::SMEM_BYTES, st>>>(mq, mk, mv, p);
+  e = launch_pdl(prefill_tc_kernel<NT>, dim3(grid), dim3(Cfg<NT>::THREADS), Cfg<NT>::SMEM_BYTES, st, mq, mk, mv, p);
   note_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace
@@ -592,10 +596,10 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int plan_e
       !make_map(&mv, a.v, a.Hkv, total_tokens))
     return cudaErrorInvalidValue;
   if (plan_entries <= 0) return cudaSuccess;
-  prefill_plan_kernel<<<1, PLAN_THREADS, 0, st>>>(a.cu_seqlens, a.batch, (a.max_seqlen + BM - 1) / BM,
-                                                  reinterpret_cast<int4*>(plan));
+  cudaError_t e = launch_pdl(prefill_plan_kernel, dim3(1), dim3(PLAN_THREADS), 0, st, a.cu_seqlens, a.batch,
+                             (a.max_seqlen + BM - 1) / BM, reinterpret_cast<int4*>(plan));
   note_launch();
-  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   TcParams p{};
   p.o = a.o; p.lse = a.lse; p.plan = reinterpret_cast<const int4*>(plan); p.status = status_word;

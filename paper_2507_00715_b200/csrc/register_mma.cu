@@ -35,6 +35,7 @@ __global__ void __launch_bounds__(NW * 32, 12 / NW) register_mma_kernel(Register
   using G = RGeo<D>;
   constexpr int KSTEPS = D / 16, NTILES = D / 8, CH = G::ROWB / 16;
   extern __shared__ __align__(128) uint8_t smem[];
+  pdl_wait();   // everything below reads or writes global memory
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kvh = blockIdx.x, b = blockIdx.y;
   const int R = a.R, g = a.Hq / a.Hkv, n_rows = g * R;
@@ -86,6 +87,7 @@ __global__ void __launch_bounds__(NW * 32, 12 / NW) register_mma_kernel(Register
   bf16* og = reinterpret_cast<bf16*>(a.o_reg);
   cp_async_wait<0>();
   __syncthreads();   // every warp's copies have landed (warps without a tile take part too)
+  pdl_launch_dependents();
 
   for (int tile = warp; tile * 16 < n_rows; tile += NW) {
     const int rr0 = tile * 16 + (lane >> 2), rr1 = rr0 + 8;
@@ -198,9 +200,9 @@ cudaError_t launch_r(const RegisterArgs& a, cudaStream_t st) {
   cudaError_t e = ensure_dynamic_smem<register_mma_kernel<D>>(2 * MAX_R * RGeo<D>::PITCH + NW * 16 * RGeo<D>::PITCH);
   if (e != cudaSuccess) return e;
   dim3 grid(a.Hkv, a.batch);
-  register_mma_kernel<D><<<grid, NW * 32, smem, st>>>(a, r_pad);
+  e = launch_pdl(register_mma_kernel<D>, grid, dim3(NW * 32), smem, st, a, r_pad);
   note_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace
