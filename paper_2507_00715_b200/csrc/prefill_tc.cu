@@ -12,14 +12,16 @@
 //   warp 2     TMA: the Q tiles of the next item, as soon as the last S of the current item has read them
 //   warp 1     one thread issues tcgen05.mma: S_x = Q_x K^T into tensor memory, O_x += P_x V with P_x read
 //              from tensor memory; after the last P V of an item it goes straight on to the first S of the next
-//   warps 4..  one softmax warpgroup per M-tile, one query row per thread: S_x from TMEM in 32-column chunks
-//              (one pass for the row maximum, one for the exponentials), online softmax in the log2 domain,
-//              P_x written back as bf16 over the columns of S_x it has already consumed; the same warps
-//              normalise and store O_x when the item ends, while the tensor core already works on the next item
+//   warps 4..  one softmax warpgroup per M-tile, one query row per thread: S_x from TMEM in 32-column chunks,
+//              online softmax in the log2 domain in ONE pass per tile (the reference maximum of the row is the one
+//              the earlier tiles left; the first tile of an item finds its own in a pass of its own), packed
+//              fp32x2 arithmetic, P_x kept in registers until the reference is known to hold and then written as
+//              bf16 over the first 64 columns of S_x; the same warps normalise and store O_x when the item ends,
+//              while the tensor core already works on the next item
 // With two M-tiles the tensor core works on one while the other is in its softmax (S_A, S_B, O_A, O_B fill
 // the 512 TMEM columns).  The running output stays in TMEM.  The softmax reference maximum is only raised
-// when the row maximum grows by more than 2^8; then the owning warp rescales its 32 rows of O in TMEM.
-// Exact after the final division by the row sum.
+// when the row maximum grows by more than 2^8; then the owning warp rescales its 32 rows of O in TMEM and
+// redoes the tile (S_x is still intact).  Exact after the final division by the row sum.
 //
 // Every mbarrier wait is bounded; when one runs out the CTA raises its abort flag, writes
 // EARN_ERR_TIMEOUT to the status word, drains what it has in flight, frees its TMEM and returns.
@@ -95,44 +97,6 @@ __device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
       "mov.b64 {%0, %1}, rd;\n\t}"
       : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
 }
-__device__ __forceinline__ void add2s(float& d0, float& d1, float a0, float a1, float c) {   // d = a + c
-  asm("{\n\t.reg .b64 ra, rc, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rc, {%4, %4};\n\tadd.rn.ftz.f32x2 rd, ra, rc;\n\t"
-      "mov.b64 {%0, %1}, rd;\n\t}"
-      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(c));
-}
-__device__ __forceinline__ void sub2(float& d0, float& d1, float a0, float a1, float b0, float b1) {   // d = a - b
-  asm("{\n\t.reg .b64 ra, rb, rd;\n\tmov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tsub.rn.ftz.f32x2 rd, ra, rb;\n\t"
-      "mov.b64 {%0, %1}, rd;\n\t}"
-      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
-}
-__device__ __forceinline__ void fma2v(float& d0, float& d1, float b0, float b1, float c) {   // d = d * b + c
-  asm("{\n\t.reg .b64 rb, rc, rd;\n\tmov.b64 rd, {%0, %1};\n\tmov.b64 rb, {%2, %3};\n\tmov.b64 rc, {%4, %4};\n\t"
-      "fma.rn.ftz.f32x2 rd, rd, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
-      : "+f"(d0), "+f"(d1) : "f"(b0), "f"(b1), "f"(c));
-}
-
-// 2^x for a pair of lanes on the FMA pipe instead of the special-function unit: x = n + f with n = round(x),
-// f in [-1/2, 1/2]; 2^f by a cubic (relative error 7.5e-5, far below the bf16 rounding of P); the integer n is
-// added into the exponent field.  x is clamped at -126, so a masked (-inf) logit gives 2^-126, which vanishes
-// against the row sum.  Used for a fixed share of the columns so that both pipes work at the same time.
-__device__ __forceinline__ void exp2_poly2(float& e0, float& e1, float x0, float x1) {
-  constexpr float MAGIC = 12582912.f;   // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
-  x0 = fmaxf(x0, -126.f);
-  x1 = fmaxf(x1, -126.f);
-  float t0, t1, n0, n1, f0, f1, p0, p1;
-  add2s(t0, t1, x0, x1, MAGIC);
-  add2s(n0, n1, t0, t1, -MAGIC);
-  sub2(f0, f1, x0, x1, n0, n1);
-  fma2(p0, p1, f0, f1, 0.055171460f, 0.24261086f);
-  fma2v(p0, p1, f0, f1, 0.69326097f);
-  fma2v(p0, p1, f0, f1, 0.99992812f);
-  e0 = __uint_as_float(__float_as_uint(p0) + (__float_as_uint(t0) << 23));
-  e1 = __uint_as_float(__float_as_uint(p1) + (__float_as_uint(t1) << 23));
-}
-#ifndef EARN_POLY_MASK
-#define EARN_POLY_MASK 0x5252u   // which of the 16 column pairs of a 32-column chunk take the polynomial (6 of 16)
-#endif
-
 template <int NT>
 __global__ void __launch_bounds__(Cfg<NT>::THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -406,12 +370,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 mx = max3(mx, s0, s1);
                 float e0, e1;
                 fma2(e0, e1, s0, s1, sl2, neg_m);
-                if ((EARN_POLY_MASK >> (c >> 1)) & 1u) {
-                  exp2_poly2(e0, e1, e0, e1);
-                } else {
-                  e0 = ex2(e0);
-                  e1 = ex2(e1);
-                }
+                e0 = ex2(e0);   // all on the special-function unit: moving a share of them to a cubic on the FMA pipe
+                e1 = ex2(e1);   // made the kernel slower on B200 (731 us -> 758 us per 7B layer at 6 of 16 pairs)
                 add2(ls0, ls1, e0, e1);
                 pk[q][c >> 1] = pack_bf16(e0, e1);
               }

@@ -92,8 +92,7 @@ __global__ void __launch_bounds__(NW * 32, 12 / NW) register_mma_kernel(Register
   for (int tile = warp; tile * 16 < n_rows; tile += NW) {
     const int rr0 = tile * 16 + (lane >> 2), rr1 = rr0 + 8;
     // row -> (head in group, register index); rows past g*R read nothing and write nothing
-    const int gi0 = rr0 / R, m0r = rr0 % R, gi1 = rr1 / R, m1r = rr1 % R;
-    const bool ok0 = rr0 < n_rows, ok1 = rr1 < n_rows;
+    const int m0r = rr0 % R, m1r = rr1 % R;
     if (tile != warp) {   // later tiles of this warp: the first one came in with the K/V rows
       tile_off = row_offset(tile);
       load_q_tile(tile_off);
