@@ -23,6 +23,8 @@
 // Online softmax in the log2 domain.  With a single split the CTA writes O itself; otherwise it writes a
 // normalised partial + log2-domain LSE, takes a ticket, and the CTA holding the last ticket of its
 // (sequence, kv head, row tile) folds the partials -- one launch, and no CTA ever waits for another.
+// The fold is on the critical path of the launch (it starts when the slowest split ends), so it walks the
+// splits once with a running maximum, four splits' loads in flight at a time.
 #include "earn_common.cuh"
 #include "mma_sync.cuh"
 #include "sm100_ptx.cuh"
@@ -61,9 +63,11 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   pdl_wait();   // everything below reads or writes global memory
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b = blockIdx.z, kvh = blockIdx.y;
+  // kv heads vary fastest over the grid: the CTAs that read the same rows of the packed K/V tensors (one 256-byte
+  // slice each of a 2 KB row) start next to each other and walk those rows together
+  const int b = blockIdx.z, kvh = blockIdx.x;
   const int row_tiles = a.plan.row_tiles;
-  const int split = blockIdx.x / row_tiles, row0 = (blockIdx.x % row_tiles) * 16;
+  const int split = blockIdx.y / row_tiles, row0 = (blockIdx.y % row_tiles) * 16;
   const int g = a.Hq / a.Hkv, W = a.beams, n_rows = W * g, step = a.step;
   const int seq_lo = a.src.paged ? 0 : a.cu_seqlens[b];
   const int shared_len = a.src.paged ? a.src.n_regs : (a.cu_seqlens[b + 1] - seq_lo);
@@ -310,6 +314,99 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
     return;
   }
 
+  if (NWARPS == 1) {
+    // ---- split-KV, one warp: publish this split's normalised partial rows straight from the accumulator
+    // fragments, take a ticket, and let the warp that holds the last ticket of its (sequence, kv head, row tile)
+    // fold all partials.  No CTA waits for another.  The fold walks the splits once, four at a time with all
+    // their loads in flight together, keeping a running maximum (what one thread per row walking the splits in
+    // two passes cost: 6 to 13 us of L2 round trips at 8 to 13 splits).
+    const int r0 = lane >> 2, r1 = r0 + 8;
+    const int64_t prow0 = ((int64_t)(b * a.Hkv + kvh) * a.plan.n_splits + split) * a.plan.rows_pad + row0;
+    {
+      const float i0 = 1.f / l0, i1 = 1.f / l1;
+      float* p0 = a.part_o + (prow0 + r0) * D + c2;
+      float* p1 = a.part_o + (prow0 + r1) * D + c2;
+      if (row0 + r0 < n_rows) {
+#pragma unroll
+        for (int n = 0; n < NTILES; ++n) *reinterpret_cast<float2*>(p0 + n * 8) = make_float2(o[n][0] * i0, o[n][1] * i0);
+        if ((lane & 3) == 0) a.part_lse[prow0 + r0] = m0 + log2f(l0);
+      }
+      if (row0 + r1 < n_rows) {
+#pragma unroll
+        for (int n = 0; n < NTILES; ++n) *reinterpret_cast<float2*>(p1 + n * 8) = make_float2(o[n][2] * i1, o[n][3] * i1);
+        if ((lane & 3) == 0) a.part_lse[prow0 + r1] = m1 + log2f(l1);
+      }
+    }
+    __threadfence();
+    __syncwarp();
+    const int live_splits = max(1, min(a.plan.n_splits, (shared_len + a.plan.chunk - 1) / a.plan.chunk));
+    int last = 0;
+    if (lane == 0) {
+      int32_t* ticket = a.tickets + ((int64_t)(b * a.Hkv + kvh) * row_tiles + blockIdx.y % row_tiles);
+      const int t = atomicAdd(ticket, 1);
+      last = (t == live_splits - 1);
+      if (last) *ticket = 0;   // ready for the next launch on this stream
+    }
+    if (!__shfl_sync(0xffffffffu, last, 0)) return;
+    __threadfence();
+    constexpr int V4 = D / 4, RPP = 4 * 32 / V4;   // float4 per row; rows per pass (4 float4 per lane)
+    const int live_rows = min(16, n_rows - row0);
+    const int64_t fold0 = (int64_t)(b * a.Hkv + kvh) * a.plan.n_splits * a.plan.rows_pad + row0;   // split 0, first row
+    bf16* og = reinterpret_cast<bf16*>(a.o);
+    for (int rbase = 0; rbase < live_rows; rbase += RPP) {
+      float4 acc[4];
+      float mx[4], den[4];
+      int rk[4], ck[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int idx = lane + 32 * k;
+        rk[k] = rbase + idx / V4;
+        ck[k] = idx % V4;
+        acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        mx[k] = -INFINITY;
+        den[k] = 0.f;
+      }
+      for (int s0 = 0; s0 < live_splits; s0 += 4) {
+        float lse_b[4][4];
+        float4 x_b[4][4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const bool ok = s0 + u < live_splits && rk[k] < live_rows;
+            const int64_t prow = fold0 + (int64_t)(s0 + u) * a.plan.rows_pad + rk[k];
+            lse_b[u][k] = ok ? __ldcg(a.part_lse + prow) : -INFINITY;
+            x_b[u][k] = ok ? __ldcg(reinterpret_cast<const float4*>(a.part_o + prow * D) + ck[k]) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float mn = fmaxf(mx[k], lse_b[u][k]);
+            const float sc = mn == -INFINITY ? 1.f : exp2f(mx[k] - mn), wt = mn == -INFINITY ? 0.f : exp2f(lse_b[u][k] - mn);
+            acc[k].x = acc[k].x * sc + wt * x_b[u][k].x;
+            acc[k].y = acc[k].y * sc + wt * x_b[u][k].y;
+            acc[k].z = acc[k].z * sc + wt * x_b[u][k].z;
+            acc[k].w = acc[k].w * sc + wt * x_b[u][k].w;
+            den[k] = den[k] * sc + wt;
+            mx[k] = mn;
+          }
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (rk[k] < live_rows) {
+          const int rr = row0 + rk[k];
+          const float inv = 1.f / den[k];
+          uint2 v;
+          v.x = pack2(acc[k].x * inv, acc[k].y * inv);
+          v.y = pack2(acc[k].z * inv, acc[k].w * inv);
+          *reinterpret_cast<uint2*>(og + (((int64_t)b * W + rr / g) * a.Hq + kvh * g + rr % g) * D + ck[k] * 4) = v;
+        }
+      }
+    }
+    return;
+  }
+
   float* mo = reinterpret_cast<float*>(smem);                 // [NWARPS][16][D]
   float* ml = mo + NWARPS * 16 * D;                           // [NWARPS][16][2] = (m, l)
   {
@@ -376,7 +473,7 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
     __threadfence();
     __syncthreads();
     int* is_last = reinterpret_cast<int*>(ml + NWARPS * 16 * 2);
-    int32_t* ticket = a.tickets + ((int64_t)(b * a.Hkv + kvh) * row_tiles + blockIdx.x % row_tiles);
+    int32_t* ticket = a.tickets + ((int64_t)(b * a.Hkv + kvh) * row_tiles + blockIdx.y % row_tiles);
     const int live_splits = max(1, min(a.plan.n_splits, (shared_len + a.plan.chunk - 1) / a.plan.chunk));
     if (threadIdx.x == 0) {
       const int t = atomicAdd(ticket, 1);
@@ -386,33 +483,42 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
     __syncthreads();
     if (!*is_last) return;
     __threadfence();
-    if (rr < n_rows) {
-      const int64_t prow0 = (int64_t)(b * a.Hkv + kvh) * a.plan.n_splits * a.plan.rows_pad + rr;
-      float top = -INFINITY;
-      for (int s = 0; s < live_splits; ++s) top = fmaxf(top, __ldcg(a.part_lse + prow0 + (int64_t)s * a.plan.rows_pad));
-      float den = 0.f, out[COLS];
-#pragma unroll
-      for (int c = 0; c < COLS; ++c) out[c] = 0.f;
+    // Fold: every thread of the CTA works on the valid rows of the tile (W*g is often 4 or 6 of the 16), a
+    // float4 at a time, with the loads of several splits in flight at once -- one thread per row walking the
+    // splits one after the other cost about 10 us of L2 round trips at 8 to 13 splits.
+    __syncthreads();   // `mo` / `ml` are free again
+    constexpr int NT = NWARPS * 32, V4 = D / 4;
+    const int live_rows = min(16, n_rows - row0);
+    const int64_t prow0 = (int64_t)(b * a.Hkv + kvh) * a.plan.n_splits * a.plan.rows_pad + row0;
+    float* top_s = mo;          // [16] row maximum of the split LSEs
+    float* inv_s = mo + 16;     // [16] 1 / sum of the split weights
+    for (int r = threadIdx.x; r < live_rows; r += NT) {
+      float top = -INFINITY, den = 0.f;
+#pragma unroll 8
+      for (int s = 0; s < live_splits; ++s) top = fmaxf(top, __ldcg(a.part_lse + prow0 + (int64_t)s * a.plan.rows_pad + r));
+#pragma unroll 8
+      for (int s = 0; s < live_splits; ++s) den += exp2f(__ldcg(a.part_lse + prow0 + (int64_t)s * a.plan.rows_pad + r) - top);
+      top_s[r] = top;
+      inv_s[r] = 1.f / den;
+    }
+    __syncthreads();
+    bf16* og = reinterpret_cast<bf16*>(a.o);
+    for (int idx = threadIdx.x; idx < live_rows * V4; idx += NT) {
+      const int r = idx / V4, c4 = idx % V4, rr = row0 + r;
+      const float top = top_s[r];
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
       for (int s = 0; s < live_splits; ++s) {
-        const int64_t prow = prow0 + (int64_t)s * a.plan.rows_pad;
+        const int64_t prow = prow0 + (int64_t)s * a.plan.rows_pad + r;
         const float wt = exp2f(__ldcg(a.part_lse + prow) - top);
-        den += wt;
-        const float4* po = reinterpret_cast<const float4*>(a.part_o + prow * D + cg);
-#pragma unroll
-        for (int c = 0; c < COLS; c += 4) {
-          const float4 x = __ldcg(po + c / 4);
-          out[c] += wt * x.x; out[c + 1] += wt * x.y; out[c + 2] += wt * x.z; out[c + 3] += wt * x.w;
-        }
+        const float4 x = __ldcg(reinterpret_cast<const float4*>(a.part_o + prow * D) + c4);
+        acc.x += wt * x.x; acc.y += wt * x.y; acc.z += wt * x.z; acc.w += wt * x.w;
       }
-      const float inv = 1.f / den;
-      bf16* dst = reinterpret_cast<bf16*>(a.o) + (((int64_t)b * W + rr / g) * a.Hq + kvh * g + rr % g) * D + cg;
-#pragma unroll
-      for (int c = 0; c < COLS; c += 8) {
-        uint4 v;
-        v.x = pack2(out[c] * inv, out[c + 1] * inv); v.y = pack2(out[c + 2] * inv, out[c + 3] * inv);
-        v.z = pack2(out[c + 4] * inv, out[c + 5] * inv); v.w = pack2(out[c + 6] * inv, out[c + 7] * inv);
-        *reinterpret_cast<uint4*>(dst + c) = v;
-      }
+      const float inv = inv_s[r];
+      uint2 v;
+      v.x = pack2(acc.x * inv, acc.y * inv);
+      v.y = pack2(acc.z * inv, acc.w * inv);
+      *reinterpret_cast<uint2*>(og + (((int64_t)b * W + rr / g) * a.Hq + kvh * g + rr % g) * D + c4 * 4) = v;
     }
   }
 }
@@ -423,7 +529,7 @@ cudaError_t launch_d(const DecodeArgs& a, cudaStream_t st) {
   cudaError_t e = ensure_dynamic_smem<decode_mma_kernel<D, ST, NWARPS>>(smem);
   if (e != cudaSuccess) return e;
   const int splits = a.plan.n_splits > 0 ? a.plan.n_splits : 1;
-  dim3 grid(splits * a.plan.row_tiles, a.Hkv, a.batch);
+  dim3 grid(a.Hkv, splits * a.plan.row_tiles, a.batch);
   e = launch_pdl(decode_mma_kernel<D, ST, NWARPS>, grid, dim3(NWARPS * 32), smem, st, a);
   note_launch();
   return e != cudaSuccess ? e : cudaGetLastError();

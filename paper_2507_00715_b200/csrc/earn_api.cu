@@ -56,10 +56,14 @@ DecodePlan make_decode_plan(const earn_model_t& m, const earn_batch_t& b, int be
   p.row_tiles = (p.rows + kDecodeRows - 1) / kDecodeRows;
   p.rows_pad = p.row_tiles * kDecodeRows;
   if (max_shared_len <= 0 || b.batch == 0) { p.chunk = 64; p.n_splits = 0; return p; }
-  // Split only while the unsplit CTAs would leave resident slots empty (six decode CTAs fit an SM): on B200
-  // every extra split of the 7B shapes cost time (50.9 us unsplit, 65.8 us in two splits).
+  // Split only while the unsplit CTAs would leave the GPU short of work.  Measured on B200 (8 sequences of 4096
+  // tokens, 8 kv heads): filling 4 CTA slots per SM took 32 us per layer, 6 slots 35 us, 8 slots 40 us, 3 slots
+  // 45 us -- every split adds a partial to write and fold; at the 7B shapes (512 unsplit CTAs) any split cost time.
   const long units = (long)b.batch * m.n_kv_heads * p.row_tiles;
-  const long slots = 6L * 148;
+#ifndef EARN_DECODE_SLOTS_PER_SM
+#define EARN_DECODE_SLOTS_PER_SM 4
+#endif
+  const long slots = (long)EARN_DECODE_SLOTS_PER_SM * 148;
   long splits = slots / units;
   long max_splits = (max_shared_len + 63) / 64;
   if (splits > max_splits) splits = max_splits;
