@@ -1,0 +1,166 @@
+// Decode attention (Eq. 4) when the query rows of a (sequence, kv head) fill several 16-row tiles: beam search,
+// where W beams x g heads of the group share one kv head (the paper generates with beam 20, Appendix A.3).
+//
+// Every row tile needs the whole shared segment (the prompt K/V of a layer l < k, or the compact register pages
+// of a layer l >= k).  One CTA per row tile would fetch it once per tile (three times at 10 beams x 4 heads,
+// which left the prompt-cache layers L2-bound at 2.7 TB/s on B200).  Here one CTA = (sequence, kv head, split of
+// the shared segment, group of RT row tiles), one warp per row tile:
+//   phase 1  all warps copy the shared segment tile by tile into ONE ring of shared memory (16-byte cp.async,
+//            a block-wide barrier per tile) and each warp attends its own 16 rows to every tile;
+//   phase 2  (split 0) each warp walks the generated tokens of its own beams alone, through its slice of the ring;
+//   finish   per warp, exactly as in the one-row-tile kernel: write the rows, or publish a partial and fold.
+// DRAM traffic of a prompt-cache layer of the ragged 10-beam workload fell to 737 MB (710 MB algorithmic) and the
+// layer from 260 us to 232 us; what bounds it now is latency at three CTAs per SM (166 registers per thread):
+// 40 query rows per kv head are 10 times the mma.sync work per byte of the one-beam case.  Forcing four CTAs per
+// SM (128 registers, a shallower ring) measured 271 us, two CTAs 271 us.
+#include "decode_tile.cuh"
+#include "sm100_ptx.cuh"
+
+namespace earn {
+namespace {
+using namespace dec;
+
+template <int D, int RT, int ST>   // RT warps = row tiles per CTA; ST ring stages, a multiple of RT
+__global__ void __launch_bounds__(RT * 32) decode_rows_kernel(DecodeArgs a) {
+  using G = Geo<D>;
+  constexpr int NT = RT * 32, CH = G::CH, SPW = ST / RT;   // SPW: ring stages a warp owns in phase 2
+  static_assert(ST % RT == 0 && SPW >= 1 && NT % CH == 0, "ring slices");
+  extern __shared__ __align__(128) uint8_t smem[];
+  pdl_wait();   // everything below reads or writes global memory
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int b = blockIdx.z, kvh = blockIdx.x;
+  const int row_groups = (a.plan.row_tiles + RT - 1) / RT;
+  const int split = blockIdx.y / row_groups, row_tile = (blockIdx.y % row_groups) * RT + warp;
+  const bool active = row_tile < a.plan.row_tiles;   // a warp without a row tile still helps with the copies
+  RowMap rm;
+  rm.b = b; rm.kvh = kvh; rm.row0 = row_tile * 16; rm.g = a.Hq / a.Hkv; rm.W = a.beams; rm.n_rows = rm.W * rm.g; rm.Hq = a.Hq;
+  const int g = rm.g, W = rm.W, step = a.step;
+  const int seq_lo = a.src.paged ? 0 : a.cu_seqlens[b];
+  const int shared_len = a.src.paged ? a.src.n_regs : (a.cu_seqlens[b + 1] - seq_lo);
+  const int key_begin = split * a.plan.chunk;
+  const int n_shared = max(min(key_begin + a.plan.chunk, shared_len) - key_begin, 0);
+  if (n_shared == 0 && split != 0) return;   // a split past the end of this sequence
+  const int n_sh_tiles = (n_shared + KT - 1) / KT;
+  const float scale_log2 = a.scale * kLog2e;
+
+  Sources src;
+  src.k[0] = reinterpret_cast<const bf16*>(a.src.k); src.v[0] = reinterpret_cast<const bf16*>(a.src.v);
+  src.k[1] = reinterpret_cast<const bf16*>(a.k_priv); src.v[1] = reinterpret_cast<const bf16*>(a.v_priv);
+  src.k[2] = reinterpret_cast<const bf16*>(a.k_new); src.v[2] = reinterpret_cast<const bf16*>(a.v_new);
+
+  // ---- phase 1 copies: thread -> (row r_t + i * NT/CH of the tile, 16-byte chunk c_t), K and V alike
+  const uint32_t ring = ptx::smem_u32(smem);
+  const int c_t = threadIdx.x % CH, r_t = threadIdx.x / CH;
+  const bool affine = !a.src.paged || a.src.block_table == nullptr;
+  const int64_t row_base = a.src.paged ? (int64_t)b * a.src.pages_per_seq * EARN_PAGE_TOKENS : (int64_t)seq_lo;
+  auto issue_shared = [&](int tile, int stage) {
+    const uint32_t kdst = ring + stage * G::STAGE_B + (uint32_t)c_t * 16, vdst = kdst + G::TILE_B;
+#pragma unroll
+    for (int i = 0; i < KT * CH / NT; ++i) {
+      const int r = r_t + i * (NT / CH), p = tile * KT + r;
+      const bool ok = p < n_shared;
+      const int64_t row = !ok ? 0 : affine ? row_base + key_begin + p : key_row(a.src, b, key_begin + p);
+      const int64_t off = (row * a.Hkv + kvh) * D + c_t * 8;
+      cp_async16(kdst + r * G::PITCH, src.k[0] + off, ok ? 16 : 0);
+      cp_async16(vdst + r * G::PITCH, src.v[0] + off, ok ? 16 : 0);
+    }
+  };
+#pragma unroll
+  for (int s = 0; s < ST - 1; ++s) {
+    if (s < n_sh_tiles) issue_shared(s, s);
+    cp_async_commit();
+  }
+
+  // ---- Eq. 4: append (split 0), and the Q fragments, while the first tiles are in flight
+  RowTile<D> t;
+  if (active) {
+    if (split == 0) append_new_rows<D>(a, rm, lane, 32);
+    t.init(reinterpret_cast<const bf16*>(a.q), rm, lane);
+  }
+
+  for (int it = 0; it < n_sh_tiles; ++it) {
+    cp_async_wait<ST - 2>();   // this thread's copies of tile `it` have landed ...
+    __syncthreads();           // ... and everyone's; every warp is also done with tile it-1, whose stage is refilled next
+    {
+      const int nxt = it + ST - 1;
+      if (nxt < n_sh_tiles) issue_shared(nxt, nxt % ST);
+      cp_async_commit();
+    }
+    if (active) {
+      const uint32_t ks = ring + (it % ST) * G::STAGE_B, vs = ks + G::TILE_B;
+      t.attend(ks, vs, scale_log2, lane, (it + 1) * KT > n_shared, [&](int c, bool) { return it * KT + c < n_shared; });
+    }
+  }
+  cp_async_wait<0>();
+  pdl_launch_dependents();   // from here on the next kernel on the stream may be scheduled
+  __syncthreads();           // the ring is idle: each warp takes its slice
+  if (!active) return;
+
+  // ---- phase 2 (split 0): the generated tokens of this row tile's beams, newest from k_new / v_new
+  if (split == 0) {
+    const int w_lo = rm.row0 / g, w_hi = min((rm.row0 + 15) / g, W - 1);
+    const int n_priv = (w_hi - w_lo + 1) * step, n_pt = (n_priv + KT - 1) / KT;
+    const int beam0 = (rm.row0 + (lane >> 2)) / g, beam1 = (rm.row0 + (lane >> 2) + 8) / g;
+    const uint32_t mine = ring + warp * SPW * G::STAGE_B;
+    auto issue_private = [&](int tile, int stage) {
+      const int pk = tile * KT + lane;
+      int64_t off = -1;
+      int which = 1;
+      if (lane < KT && pk < n_priv) off = private_row<D>(a, b, kvh, w_lo, pk, which);
+      copy_resolved_tile<D>(mine + stage * G::STAGE_B, off, which, src, lane);
+    };
+#pragma unroll
+    for (int s = 0; s < SPW - 1; ++s) {
+      if (s < n_pt) issue_private(s, s);
+      cp_async_commit();
+    }
+    for (int it = 0; it < n_pt; ++it) {
+      {
+        const int nxt = it + SPW - 1;
+        if (nxt < n_pt) issue_private(nxt, nxt % SPW);
+        cp_async_commit();
+        cp_async_wait<SPW - 1>();
+        __syncwarp();
+      }
+      const uint32_t ks = mine + (it % SPW) * G::STAGE_B, vs = ks + G::TILE_B;
+      t.attend(ks, vs, scale_log2, lane, true, [&](int c, bool second) {   // only the row's own beam is visible
+        const int pk = it * KT + c;
+        return pk < n_priv && (w_lo + pk / step) == (second ? beam1 : beam0);
+      });
+      __syncwarp();
+    }
+    cp_async_wait<0>();
+    __syncwarp();
+  }
+
+  t.reduce_sums();
+  if (a.plan.n_splits <= 1) {
+    t.store_rows(smem + warp * SPW * G::STAGE_B, reinterpret_cast<bf16*>(a.o), rm, lane);
+  } else {
+    const int live_splits = max(1, min(a.plan.n_splits, (shared_len + a.plan.chunk - 1) / a.plan.chunk));
+    publish_and_fold<D>(t, a, rm, split, live_splits, row_tile, lane);
+  }
+}
+
+template <int D, int RT, int ST>
+cudaError_t launch_rows(const DecodeArgs& a, cudaStream_t st) {
+  constexpr int smem = ST * Geo<D>::STAGE_B;
+  cudaError_t e = ensure_dynamic_smem<decode_rows_kernel<D, RT, ST>>(smem);
+  if (e != cudaSuccess) return e;
+  const int splits = a.plan.n_splits > 0 ? a.plan.n_splits : 1;
+  dim3 grid(a.Hkv, splits * ((a.plan.row_tiles + RT - 1) / RT), a.batch);
+  e = launch_pdl(decode_rows_kernel<D, RT, ST>, grid, dim3(RT * 32), smem, st, a);
+  note_launch();
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_decode_rows(const DecodeArgs& a, cudaStream_t st) {
+  const bool two = a.plan.row_tiles == 2;
+  if (a.D == 64) return two ? launch_rows<64, 2, 6>(a, st) : launch_rows<64, 4, 8>(a, st);
+  return two ? launch_rows<128, 2, 6>(a, st) : launch_rows<128, 4, 8>(a, st);
+}
+
+}  // namespace earn

@@ -59,7 +59,8 @@ DecodePlan make_decode_plan(const earn_model_t& m, const earn_batch_t& b, int be
   // Split only while the unsplit CTAs would leave the GPU short of work.  Measured on B200 (8 sequences of 4096
   // tokens, 8 kv heads): filling 4 CTA slots per SM took 32 us per layer, 6 slots 35 us, 8 slots 40 us, 3 slots
   // 45 us -- every split adds a partial to write and fold; at the 7B shapes (512 unsplit CTAs) any split cost time.
-  const long units = (long)b.batch * m.n_kv_heads * p.row_tiles;
+  // CTAs per split: one per (sequence, kv head) and group of row tiles (up to four row tiles share a CTA)
+  const long units = (long)b.batch * m.n_kv_heads * (p.row_tiles <= 2 ? 1 : (p.row_tiles + 3) / 4);
 #ifndef EARN_DECODE_SLOTS_PER_SM
 #define EARN_DECODE_SLOTS_PER_SM 4
 #endif

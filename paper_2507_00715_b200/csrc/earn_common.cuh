@@ -139,6 +139,8 @@ struct DecodeArgs {
 cudaError_t launch_decode_simt(const DecodeArgs& a, cudaStream_t st);   // fp32 debug path
 // bf16: cp.async ring + mma.sync; max_shared_len = longest shared segment of the batch (picks the ring depth)
 cudaError_t launch_decode_mma(const DecodeArgs& a, int max_shared_len, cudaStream_t st);
+// bf16, several row tiles (beams x group size > 16): the row tiles of a CTA share one pass over the shared segment
+cudaError_t launch_decode_rows(const DecodeArgs& a, cudaStream_t st);
 
 struct CompactArgs {
   const void *k, *v, *q;
