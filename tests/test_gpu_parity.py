@@ -106,3 +106,14 @@ def test_batch_order_does_not_matter():
     w2 = w.replace(lens=tuple(w.lens[b] for b in order))
     o2 = make_session(w2).prefill_layer(0, pieces(q), pieces(k), pieces(v))
     assert torch.equal(o2, pieces(o))
+
+
+def test_beam_search_row_tiles_share_the_cache_pass():
+    """More query rows per kv head than one 16-row tile (beams x group size > 16): two row tiles, then five row
+    tiles in two groups with split-KV on a long prompt, scattered pages, and head_dim 64."""
+    run_workload_and_compare(BASE.replace(seed=24, n_q_heads=8, n_kv_heads=2, lens=(150, 90), batch=2, beams=5,
+                                          decode_steps=4, r_head=9, r_tail=8), paged_shuffle_seed=3)
+    run_workload_and_compare(BASE.replace(seed=25, n_q_heads=8, n_kv_heads=2, lens=(1500,), batch=1, beams=20,
+                                          decode_steps=3, r_head=16, r_tail=16, n_layers=2, split_k=1), check_lse=False)
+    run_workload_and_compare(BASE.replace(seed=26, head_dim=64, n_q_heads=8, n_kv_heads=2, lens=(200, 64), batch=2,
+                                          beams=7, decode_steps=3, r_head=4, r_tail=4))
