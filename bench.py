@@ -407,6 +407,49 @@ def profile_one_kernel(w: wl.Workload, dev, which: str, launches: int = 3):
     print(json.dumps({"profiled": which, "workload": workload_desc(w1), "launches": launches}))
 
 
+def sweep_split_layer(w: wl.Workload, dev, ks, args):
+    """The k sweep of the long-history workload (and of any other): the whole hot path timed once per split layer.
+    Section 3.3 predicts time ~ k/N of the vanilla model for prefill (Eq. 8) and a cache of kL + (N-k)r entries
+    (Eq. 9); k = N is the vanilla model.  One JSON line per k."""
+    lens = wl.seqlens(w)
+    tokens = int(lens.sum()) + w.batch * w.beams * w.decode_steps
+    base = None
+    for k in ks:
+        wk = w.replace(split_k=k)
+        job = GpuJob(wk, dev)
+        job.step()
+        torch.cuda.synchronize()
+        if not args.no_graphs:
+            job.capture_graphs()
+        for _ in range(args.warmup):
+            job.step()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            job.step(record=True)
+        e1.record()
+        torch.cuda.synchronize()
+        assert job.ses.device_status() == 0
+        t = e0.elapsed_time(e1) * 1e-3 / args.steps
+        seg = {kind: sec * n * 1e3 for kind, (sec, n, _) in job.segment_times().items()}
+        T, N = wk.decode_steps, wk.n_layers
+        earn_e, van_e = job.ses.kv_entries(T), N * (int(lens.sum()) + wk.batch * wk.beams * T)
+        L, r = float(lens.mean()), wk.n_regs
+        line = {"sweep": "split_k", "workload": workload_desc(wk), "k": k, "value": tokens / t, "unit": UNIT,
+                "ms_per_step": t * 1e3, "prefill_ms": seg.get("prefill", 0.0) + seg.get("register_layer", 0.0),
+                "decode_ms": seg.get("decode_full", 0.0) + seg.get("decode_compact", 0.0),
+                "kv_reduction_measured": 1.0 - earn_e / van_e,
+                "gamma_cache_eq9": (N - k) * (L - r) / (N * L), "k_over_N": k / N}
+        if k == N:
+            base = t
+        if base is not None:
+            line["speedup_vs_vanilla"] = base / t
+        print(json.dumps(line), flush=True)
+        del job
+        torch.cuda.empty_cache()
+
+
 def blas_threads() -> int:
     try:
         import threadpoolctl
@@ -431,6 +474,9 @@ def main():
     ap.add_argument("--profile-kernel", default=None,
                     choices=["prefill", "compact", "register", "decode_compact", "decode_full"],
                     help="small case for a profiler: allocate ONE layer of the workload and launch that step 3 times")
+    ap.add_argument("--sweep-k", default=None,
+                    help="comma-separated split layers k: time the workload once per k (one JSON line each, k = N is the "
+                         "vanilla model) instead of the single benchmark line")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "earn" else args.warmup
 
@@ -478,6 +524,10 @@ def main():
 
     if args.profile_kernel:
         profile_one_kernel(w, dev, args.profile_kernel)
+        return
+
+    if args.sweep_k:
+        sweep_split_layer(w, dev, [int(x) for x in args.sweep_k.split(",")], args)
         return
 
     job = GpuJob(replicas.rank_workload(w, rank), dev)

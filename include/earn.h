@@ -104,6 +104,14 @@ earn_status_t earn_workspace_init(void* workspace, size_t workspace_bytes, earn_
  * EARN_ERR_TIMEOUT if a bounded wait inside a kernel ran out since earn_workspace_init. */
 earn_status_t earn_device_status(const void* workspace, earn_stream_t stream);
 
+/* Failure-path self-test (the paper has no counterpart): launches one small kernel that waits, with the bounded
+ * wait the tensor-core kernels use, on a barrier nothing will ever complete.  After `limit_cycles` SM clocks
+ * (1 .. 2e9, i.e. at most about a second) the wait gives up, the kernel writes EARN_ERR_TIMEOUT to the workspace
+ * status word and returns normally; earn_device_status() then reports it and earn_workspace_init() clears it.
+ * The context stays usable.  Errors: limit out of range -> INVALID_ARG; workspace NULL / too small -> WORKSPACE. */
+earn_status_t earn_selftest_wait_timeout(void* workspace, size_t workspace_bytes, int64_t limit_cycles,
+                                         earn_stream_t stream);
+
 /* Step 1 — full causal attention of a layer l < k over every prompt token
  * (Section 3.2 "Full Computation Process"; Eq. 3 with the causal mask of a decoder-only model):
  *   O[i,h] = sum_{j<=i} softmax_j( Q[i,h].K[j,h/g] * scale ) V[j,h/g]   within each sequence, g = Hq/Hkv.

@@ -46,6 +46,7 @@ SYMBOLS = {
     "earn_workspace_bytes": (C.c_size_t, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32]),
     "earn_workspace_init": (C.c_int, [C.c_void_p, C.c_size_t, C.c_void_p]),
     "earn_device_status": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "earn_selftest_wait_timeout": (C.c_int, [C.c_void_p, C.c_size_t, C.c_int64, C.c_void_p]),
     "earn_prefill_attn": (C.c_int, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32, C.c_void_p, C.c_void_p,
                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "earn_compact_kv": (C.c_int, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32, C.c_void_p, C.c_void_p,
@@ -160,6 +161,11 @@ def earn_workspace_init(workspace: torch.Tensor) -> None:
 
 def earn_device_status(workspace: torch.Tensor) -> int:
     return lib().earn_device_status(_ptr(workspace), _stream())
+
+
+def earn_selftest_wait_timeout(workspace: torch.Tensor, limit_cycles: int) -> None:
+    _check(lib().earn_selftest_wait_timeout(_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                            int(limit_cycles), _stream()), "earn_selftest_wait_timeout")
 
 
 def _ws(workspace):

@@ -117,3 +117,21 @@ def test_beam_search_row_tiles_share_the_cache_pass():
                                           decode_steps=3, r_head=16, r_tail=16, n_layers=2, split_k=1), check_lse=False)
     run_workload_and_compare(BASE.replace(seed=26, head_dim=64, n_q_heads=8, n_kv_heads=2, lens=(200, 64), batch=2,
                                           beams=7, decode_steps=3, r_head=4, r_tail=4))
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_survives():
+    """Failure detection without a fault: a bounded device-side wait on a barrier nothing completes gives up after
+    its limit, the kernel returns normally with EARN_ERR_TIMEOUT in the status word, and the library keeps working."""
+    from paper_2507_00715_b200 import binding as B
+    from parity_util import make_session
+
+    w = BASE.replace(seed=27, lens=(200, 140), batch=2, n_layers=1, split_k=1, decode_steps=0)
+    ses = make_session(w)
+    assert ses.device_status() == B.EARN_OK
+    B.earn_selftest_wait_timeout(ses.workspace, 2_000_000)          # about a millisecond
+    assert ses.device_status() == B.EARN_ERR_TIMEOUT
+    B.earn_workspace_init(ses.workspace)
+    assert ses.device_status() == B.EARN_OK
+    run_workload_and_compare(w)                                      # the context is still usable
+    with pytest.raises(B.EarnError):
+        B.earn_selftest_wait_timeout(ses.workspace, 10**12)          # limit beyond a second: refused on the host
