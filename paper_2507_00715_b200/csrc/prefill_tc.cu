@@ -20,8 +20,9 @@
 //              while the tensor core already works on the next item
 // With two M-tiles the tensor core works on one while the other is in its softmax (S_A, S_B, O_A, O_B fill
 // the 512 TMEM columns).  The running output stays in TMEM.  The softmax reference maximum is only raised
-// when the row maximum grows by more than 2^8; then the owning warp rescales its 32 rows of O in TMEM and
-// redoes the tile (S_x is still intact).  Exact after the final division by the row sum.
+// when a tile's sum of exponentials exceeds 2^8 (no term can exceed that bound otherwise); then the owning warp
+// rescales its 32 rows of O in TMEM and redoes the tile (S_x is still intact).  Exact after the final division
+// by the row sum.
 //
 // Every mbarrier wait is bounded; when one runs out the CTA raises its abort flag, writes
 // EARN_ERR_TIMEOUT to the status word, drains what it has in flight, frees its TMEM and returns.
@@ -38,7 +39,6 @@ constexpr int BM = 128, BN = 128, HD = 128;
 constexpr int TILE = BM * HD * 2;   // bytes of one 128 x 128 bf16 tile
 constexpr int HALF = TILE / 2;      // one 64-column block of it (128 rows x 128 B)
 constexpr long long WAIT_LIMIT = 2000000000LL;     // about one second of SM clocks
-constexpr float RESCALE_THRESHOLD = 8.f;           // log2 units
 
 template <int NT>
 struct Cfg {
@@ -308,8 +308,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const bool diag = j == it.n_tiles - 1;        // key column c of this tile is visible to row r iff c <= r
         const int n_chunks = diag ? wq + 1 : 4;       // 32-column chunks with a visible key for this warp's rows
         uint32_t a[32], b[32], pk[4][16];
-        if (j == 0) {
-          // ---- first tile of the item: the reference is its own row maximum, found in a pass of its own
+        // row maximum of the visible part of S_x(j), scaled into the log2 domain (a pass of its own over TMEM)
+        auto row_max = [&]() {
           float mx = -INFINITY;
           tmem_ld_32x32(t_s, a);
           if (n_chunks > 1) tmem_ld_32x32(t_s + 32, b);
@@ -339,17 +339,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
               tmem_wait_ld(b);
             }
           }
-          m_ref = mx * sl2;
-        }
-        // ---- P = 2^(S * scale - m_ref) as bf16 pairs (kept in registers until the reference is known to hold),
-        //      row sum and row maximum in the same pass.  If the maximum outgrew the reference by more than the
-        //      threshold (rare: the reference already covers every earlier tile), raise it, rescale what has been
-        //      accumulated, and redo the pass; S_x is still intact because nothing has been written over it.
+          return mx * sl2;
+        };
+        if (j == 0) m_ref = row_max();   // first tile of the item: the reference is its own row maximum
+        // ---- P = 2^(S * scale - m_ref) as bf16 pairs (kept in registers until the reference is known to hold) and
+        //      their row sum, in one pass.  The reference is the one earlier tiles left.  If this tile's sum of
+        //      exponentials exceeds 2^8 some logit may have outgrown the reference by more than the threshold
+        //      (rare: with the reference at the running maximum every term is <= 1 and the sum <= 128): then find
+        //      the tile's own maximum, raise the reference, rescale what has been accumulated, and redo the pass.
+        //      S_x is still intact because nothing has been written over it.  No term ever exceeds 2^8.
         float ls0, ls1;
 #pragma unroll 1
         for (int attempt = 0;; ++attempt) {
           const float neg_m = -m_ref;
-          float mx = -INFINITY;
           ls0 = ls1 = 0.f;
           tmem_ld_32x32(t_s, a);
           tmem_wait_ld(a);
@@ -366,10 +368,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
               }
 #pragma unroll
               for (int c = 0; c < 32; c += 2) {
-                const float s0 = __uint_as_float(cur[c]), s1 = __uint_as_float(cur[c + 1]);
-                mx = max3(mx, s0, s1);
                 float e0, e1;
-                fma2(e0, e1, s0, s1, sl2, neg_m);
+                fma2(e0, e1, __uint_as_float(cur[c]), __uint_as_float(cur[c + 1]), sl2, neg_m);
                 e0 = ex2(e0);   // all on the special-function unit: moving a share of them to a cubic on the FMA pipe
                 e1 = ex2(e1);   // made the kernel slower on B200 (731 us -> 758 us per 7B layer at 6 of 16 pairs)
                 add2(ls0, ls1, e0, e1);
@@ -381,12 +381,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
               for (int c = 0; c < 16; ++c) pk[q][c] = 0u;
             }
           }
-          const float mxs = mx * sl2;
-          const bool grow = mxs > m_ref + RESCALE_THRESHOLD;
+          const bool grow = !(ls0 + ls1 <= 256.f);   // also catches a sum that overflowed
           if (attempt > 0 || !__any_sync(0xffffffffu, grow)) break;
           // S_x(j) was issued after P_x V of tile j-1, so the commit that signalled it covers that too: O_x is quiescent
-          const float alpha = grow ? ex2(m_ref - mxs) : 1.f;
-          if (grow) m_ref = mxs;
+          const float mxs = row_max();
+          const float alpha = mxs > m_ref ? ex2(m_ref - mxs) : 1.f;
+          m_ref = fmaxf(m_ref, mxs);
           l0 *= alpha;
           l1 *= alpha;
 #pragma unroll

@@ -135,3 +135,22 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_survives():
     run_workload_and_compare(w)                                      # the context is still usable
     with pytest.raises(B.EarnError):
         B.earn_selftest_wait_timeout(ses.workspace, 10**12)          # limit beyond a second: refused on the host
+
+
+def test_prefill_logits_that_keep_rising_take_the_rescale_path():
+    """Logits that grow along the sequence by far more than the lazy-rescale bound: every key tile after the first
+    must raise the softmax reference, rescale the running output and redo its pass."""
+    from oracle import earn_oracle as orc
+    from parity_util import assert_close, make_session, to_np
+
+    w = BASE.replace(seed=28, lens=(700, 390), batch=2, n_layers=1, split_k=1, decode_steps=0, n_q_heads=4, n_kv_heads=2)
+    cu = wl.cu_seqlens(w)
+    q, k, v = wl.layer_qkv(w.replace(sink_q_bias=False), 0, "cuda")
+    u = torch.nn.functional.normalize(torch.randn(w.head_dim, device="cuda"), dim=0)
+    pos = torch.cat([torch.arange(int(n), device="cuda") for n in wl.seqlens(w)]).float()
+    # scaled logit of key j grows by about 0.35 per position: +45 per 128-key tile, +65 in the log2 domain
+    k = (k.float() * 0.1 + (pos[:, None, None] * 0.35) * u).to(torch.bfloat16)
+    q = (q.float() * 0.1 + (w.head_dim ** 0.5) * u).to(torch.bfloat16)
+    o = make_session(w).prefill_layer(0, q, k, v)
+    ref, _ = orc.causal_attention(to_np(q), to_np(k), to_np(v), cu)
+    assert_close(o, ref, "bf16", "prefill with rising logits")
