@@ -44,9 +44,15 @@ KERNEL_SOURCES = {"prefill": "prefill_tc.cu", "compact": "compact.cu", "register
 
 
 def source_digest(fname: str) -> str:
+    """Digest of a kernel's source: the .cu file and every shared header of csrc/ (a kernel changes with either)."""
+    import glob
     import hashlib
-    with open(os.path.join(ROOT, "paper_2507_00715_b200", "csrc", fname), "rb") as f:
-        return hashlib.sha256(f.read()).hexdigest()[:12]
+    csrc = os.path.join(ROOT, "paper_2507_00715_b200", "csrc")
+    h = hashlib.sha256()
+    for path in [os.path.join(csrc, fname)] + sorted(glob.glob(os.path.join(csrc, "*.cuh"))):
+        with open(path, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:12]
 
 
 def read_traffic(name: str) -> dict:
