@@ -121,13 +121,11 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
     cp_async_commit();
   }
 
-  // ---- Eq. 4: append.  Split 0 stores the new K/V row of every beam whose first query row is in this tile.
-  if (split == 0) append_new_rows<D>(a, rm, threadIdx.x, NWARPS * 32);
-
   // ---- Q fragments, loaded while the first tiles are in flight
   RowTile<D> t;
   t.init(reinterpret_cast<const bf16*>(a.q), rm, lane);
-  const int beam0 = (row0 + (lane >> 2)) / g, beam1 = (row0 + (lane >> 2) + 8) / g;
+  // list positions of the generated tokens each of the lane's two rows may see: its own beam's `step` tokens
+  const int vis0 = n_shared + ((row0 + (lane >> 2)) / g - w_lo) * step, vis1 = n_shared + ((row0 + (lane >> 2) + 8) / g - w_lo) * step;
 
   for (int it = 0; it < n_my; ++it) {
     const int stage = it % STAGES;
@@ -142,14 +140,16 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
     const uint32_t ks = ring + stage * G::STAGE_B, vs = ks + G::TILE_B;
     // positions past the list, and generated tokens of other beams, are invisible
     t.attend(ks, vs, scale_log2, lane, (tile + 1) * KT > n_shared, [&](int c, bool second) {
-      const int p = tile * KT + c;
-      bool vis = p < n_total;
-      if (p >= n_shared) vis = vis && (w_lo + (p - n_shared) / step) == (second ? beam1 : beam0);
-      return vis;
+      const int p = tile * KT + c, v0 = second ? vis1 : vis0;
+      return p < n_shared || (p >= v0 && p < v0 + step && p < n_total);
     });
     __syncwarp();   // every lane is done with this stage before the next iteration refills it
   }
   cp_async_wait<0>();
+  // ---- Eq. 4: append.  Split 0 stores the new K/V row of every beam whose first query row is in this tile.  Nothing
+  // in this launch reads those rows (the newest token came straight from k_new / v_new), so the copy waits until
+  // here: ahead of the Q loads its load-then-store round trip delayed them by more than a microsecond.
+  if (split == 0) append_new_rows<D>(a, rm, threadIdx.x, NWARPS * 32);
   // The next kernel on the stream may be scheduled from here on (once every CTA of this grid is past its key
   // loop): releasing it earlier let its CTAs pile up on whichever SMs had room and unbalanced the next launch
   // (55 us against 50 us per prompt-cache layer at the 7B shapes).
@@ -239,17 +239,25 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, int max_shared_len, cudaStrea
   // One warp per CTA with a deep ring streams best whenever the grid covers the GPU (measured on B200 at the 7B
   // shapes: 8.9 us per compact-cache layer against 13.0 us with four warps).  A short key list on a grid of less
   // than a CTA per SM is latency-bound instead: four warps take a tile or two each (5.9 against 6.8 us at the 1.5B
-  // shapes).  A list of at most two tiles needs no deep ring either way.
+  // shapes).
   const int g = a.Hq / a.Hkv;
   const int beams_per_tile = a.beams < (16 + g - 1) / g + 1 ? a.beams : (16 + g - 1) / g + 1;
   const int max_tiles = (max_shared_len + beams_per_tile * a.step + KT - 1) / KT;
   const long ctas = (long)(a.plan.n_splits > 0 ? a.plan.n_splits : 1) * a.plan.row_tiles * a.Hkv * a.batch;
   const bool unsplit = a.plan.n_splits <= 1;
   const bool four_warps = unsplit && max_tiles <= 16 && ctas < 148;
-  const bool small = unsplit && max_tiles <= 2;
+  // a ring of n+1 stages has a whole list of n tiles in flight from the start: short lists are latency-bound and
+  // the tile that had to wait for a free stage cost about 1.5 us at the 7B shapes
+  const bool two_tiles = unsplit && max_tiles <= 2, four_tiles = unsplit && max_tiles <= 4;
   if (a.D == 64)
-    return four_warps ? launch_d<64, 2, 4>(a, st) : small ? launch_d<64, 2, 1>(a, st) : launch_d<64, EARN_DECODE_STAGES, 1>(a, st);
-  return four_warps ? launch_d<128, 2, 4>(a, st) : small ? launch_d<128, 2, 1>(a, st) : launch_d<128, EARN_DECODE_STAGES, 1>(a, st);
+    return four_warps  ? launch_d<64, 2, 4>(a, st)
+           : two_tiles ? launch_d<64, 3, 1>(a, st)
+           : four_tiles ? launch_d<64, 5, 1>(a, st)
+                        : launch_d<64, EARN_DECODE_STAGES, 1>(a, st);
+  return four_warps  ? launch_d<128, 2, 4>(a, st)
+         : two_tiles ? launch_d<128, 3, 1>(a, st)
+         : four_tiles ? launch_d<128, 5, 1>(a, st)
+                      : launch_d<128, EARN_DECODE_STAGES, 1>(a, st);
 }
 
 }  // namespace earn

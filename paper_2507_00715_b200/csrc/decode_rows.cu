@@ -72,12 +72,9 @@ __global__ void __launch_bounds__(RT * 32) decode_rows_kernel(DecodeArgs a) {
     cp_async_commit();
   }
 
-  // ---- Eq. 4: append (split 0), and the Q fragments, while the first tiles are in flight
+  // ---- the Q fragments, while the first tiles are in flight
   RowTile<D> t;
-  if (active) {
-    if (split == 0) append_new_rows<D>(a, rm, lane, 32);
-    t.init(reinterpret_cast<const bf16*>(a.q), rm, lane);
-  }
+  if (active) t.init(reinterpret_cast<const bf16*>(a.q), rm, lane);
 
   for (int it = 0; it < n_sh_tiles; ++it) {
     cp_async_wait<ST - 2>();   // this thread's copies of tile `it` have landed ...
@@ -96,12 +93,16 @@ __global__ void __launch_bounds__(RT * 32) decode_rows_kernel(DecodeArgs a) {
   pdl_launch_dependents();   // from here on the next kernel on the stream may be scheduled
   __syncthreads();           // the ring is idle: each warp takes its slice
   if (!active) return;
+  // ---- Eq. 4: append (split 0).  Nothing in this launch reads the rows it writes (the newest token comes straight
+  // from k_new / v_new), so the copy stays out of the way of the loads above.
+  if (split == 0) append_new_rows<D>(a, rm, lane, 32);
 
   // ---- phase 2 (split 0): the generated tokens of this row tile's beams, newest from k_new / v_new
   if (split == 0) {
     const int w_lo = rm.row0 / g, w_hi = min((rm.row0 + 15) / g, W - 1);
     const int n_priv = (w_hi - w_lo + 1) * step, n_pt = (n_priv + KT - 1) / KT;
-    const int beam0 = (rm.row0 + (lane >> 2)) / g, beam1 = (rm.row0 + (lane >> 2) + 8) / g;
+    // positions of its list each of the lane's two rows may see: its own beam's `step` tokens
+    const int vis0 = ((rm.row0 + (lane >> 2)) / g - w_lo) * step, vis1 = ((rm.row0 + (lane >> 2) + 8) / g - w_lo) * step;
     const uint32_t mine = ring + warp * SPW * G::STAGE_B;
     auto issue_private = [&](int tile, int stage) {
       const int pk = tile * KT + lane;
@@ -125,8 +126,8 @@ __global__ void __launch_bounds__(RT * 32) decode_rows_kernel(DecodeArgs a) {
       }
       const uint32_t ks = mine + (it % SPW) * G::STAGE_B, vs = ks + G::TILE_B;
       t.attend(ks, vs, scale_log2, lane, true, [&](int c, bool second) {   // only the row's own beam is visible
-        const int pk = it * KT + c;
-        return pk < n_priv && (w_lo + pk / step) == (second ? beam1 : beam0);
+        const int pk = it * KT + c, v0 = second ? vis1 : vis0;
+        return pk >= v0 && pk < v0 + step && pk < n_priv;
       });
       __syncwarp();
     }

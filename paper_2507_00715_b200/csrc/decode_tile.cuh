@@ -65,14 +65,22 @@ struct RowTile {
     const int c2 = (lane & 3) * 2, mat = lane >> 3;
     const uint32_t k_lane = (uint32_t)(((mat >> 1) << 3) + (lane & 7)) * PITCH + (uint32_t)(mat & 1) * 16;
     const uint32_t v_lane = (uint32_t)(((mat & 1) << 3) + (lane & 7)) * PITCH + (uint32_t)(mat >> 1) * 16;
-    float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    // two accumulator sets per 8-column block (even / odd k-steps) halve the chain of dependent MMAs
+    float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}}, s2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
-    for (int kk = 0; kk < KSTEPS; ++kk) {
-      uint32_t b0, b1, b2, b3;
+    for (int kk = 0; kk < KSTEPS; kk += 2) {
+      uint32_t b0, b1, b2, b3, c0, c1, c2_, c3;
       ldsm_x4(ks + k_lane + kk * 32, b0, b1, b2, b3);
+      ldsm_x4(ks + k_lane + (kk + 1) * 32, c0, c1, c2_, c3);
       mma_bf16(s[0], qf[kk], b0, b1);
       mma_bf16(s[1], qf[kk], b2, b3);
+      mma_bf16(s2[0], qf[kk + 1], c0, c1);
+      mma_bf16(s2[1], qf[kk + 1], c2_, c3);
     }
+#pragma unroll
+    for (int n = 0; n < 2; ++n)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) s[n][e] += s2[n][e];
     if (masked) {
 #pragma unroll
       for (int n = 0; n < 2; ++n)
