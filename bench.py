@@ -308,18 +308,50 @@ class GpuJob:
         return h2d, d2h
 
     def step_e2e(self):
+        """One pass with every input starting in pinned host memory and every output ending there.  Prefill moves
+        26 GB in and 5 GB out at the 7B shapes, so its copies run on their own streams: the inputs of layer l+1
+        arrive while layer l computes, outputs drain behind it (two output buffers alternate).  The decode copies
+        are small and stay on the compute stream."""
         w, ses = self.w, self.ses
         ses.lineage_cur = None
+        cs = torch.cuda.current_stream()
+        if not hasattr(self, "s_h2d"):
+            self.s_h2d, self.s_d2h = torch.cuda.Stream(), torch.cuda.Stream()
+            self.o_full_alt, self.o_reg_alt = torch.empty_like(self.o_full), torch.empty_like(self.o_reg)
+        start = torch.cuda.Event()
+        start.record(cs)                      # the previous pass still reads the device inputs (decode reads K/V in place)
+        self.s_h2d.wait_event(start)
+        arrived = []
+        with torch.cuda.stream(self.s_h2d):
+            for layer in range(w.n_layers):
+                for d, h in zip(self.qkv[layer], self.h_qkv[layer]):
+                    d.copy_(h, non_blocking=True)
+                e = torch.cuda.Event()
+                e.record(self.s_h2d)
+                arrived.append(e)
+        drained = {}                          # output buffer id -> event after which it may be overwritten
+        last = None
         for layer in range(w.n_layers):
-            for d, h in zip(self.qkv[layer], self.h_qkv[layer]):
-                d.copy_(h, non_blocking=True)
+            cs.wait_event(arrived[layer])
             q, k, v = self.qkv[layer]
-            if layer < w.split_k:
-                ses.prefill_layer(layer, q, k, v, out=self.o_full)
-                self.h_o_full[layer].copy_(self.o_full, non_blocking=True)
+            full = layer < w.split_k
+            out = (self.o_full, self.o_full_alt)[layer & 1] if full else (self.o_reg, self.o_reg_alt)[layer & 1]
+            if id(out) in drained:
+                cs.wait_event(drained[id(out)])
+            if full:
+                ses.prefill_layer(layer, q, k, v, out=out)
+                host = self.h_o_full[layer]
             else:
-                ses.prefill_layer(layer, q, k, v, out=self.o_reg, q_reg=self.q_reg)
-                self.h_o_reg[layer - w.split_k].copy_(self.o_reg, non_blocking=True)
+                ses.prefill_layer(layer, q, k, v, out=out, q_reg=self.q_reg)
+                host = self.h_o_reg[layer - w.split_k]
+            done = torch.cuda.Event()
+            done.record(cs)
+            self.s_d2h.wait_event(done)
+            with torch.cuda.stream(self.s_d2h):
+                host.copy_(out, non_blocking=True)
+                last = torch.cuda.Event()
+                last.record(self.s_d2h)
+            drained[id(out)] = last
         for s in range(1, w.decode_steps + 1):
             ses.begin_step(s, self.parents[s - 1])
             for layer in range(w.n_layers):
@@ -328,6 +360,8 @@ class GpuJob:
                 q, k, v = self.dec[s - 1][layer]
                 ses.decode_layer(layer, s, q, k, v, out=self.o_dec)
                 self.h_o_dec[s - 1, layer].copy_(self.o_dec, non_blocking=True)
+        if last is not None:
+            cs.wait_event(last)               # the pass ends when its last output has reached the host
 
 
 # ------------------------------------------------------------------------------------------------
