@@ -85,7 +85,7 @@ static size_t ticket_bytes(const earn_model_t& m, const earn_batch_t& b, const D
 
 size_t prefill_plan_bytes(const earn_batch_t& b) {
   if (b.batch <= 0 || b.cu_seqlens_host == nullptr) return 0;
-  return round_up(sizeof(int4) * (size_t)prefill_plan_entries(b), 256);
+  return round_up(sizeof(int4) * (size_t)prefill_plan_entries(b, 128), 256);   // an upper bound for either block size
 }
 
 size_t workspace_head_bytes(const earn_model_t& m, const earn_batch_t& b, int beams) {
@@ -183,7 +183,8 @@ earn_status_t earn_prefill_attn(const earn_model_t* model, const earn_batch_t* b
   a.scale = scale_of(model);
   if (prefill_tc_supported(a, batch->total_tokens)) {
     if (!aligned16(workspace) || workspace_bytes < kStatusBytes + prefill_plan_bytes(*batch)) return EARN_ERR_WORKSPACE;
-    return launch_prefill_tc(a, batch->total_tokens, prefill_plan_entries(*batch),
+    return launch_prefill_tc(a, batch->total_tokens,
+                             prefill_plan_entries(*batch, prefill_rows_per_entry(model->n_q_heads, model->n_kv_heads)),
                              reinterpret_cast<char*>(workspace) + kStatusBytes, reinterpret_cast<int32_t*>(workspace),
                              (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
   }

@@ -106,7 +106,8 @@ struct PrefillArgs {
 cudaError_t launch_prefill_simt(const PrefillArgs& a, cudaStream_t st);
 // tensor-core path (bf16, head_dim 128); status_word receives EARN_ERR_TIMEOUT if a bounded wait runs out
 bool prefill_tc_supported(const PrefillArgs& a, int total_tokens);
-int prefill_plan_entries(const earn_batch_t& b);   // (sequence, 128-row query tile) pairs of the batch
+int prefill_rows_per_entry(int n_q_heads, int n_kv_heads);   // query rows one plan entry covers: 128 or 256
+int prefill_plan_entries(const earn_batch_t& b, int rows);   // (sequence, block of `rows` query rows) pairs of the batch
 // plan: device scratch of 16 bytes per plan entry, filled by a planning kernel launched ahead of the main one
 cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int plan_entries, void* plan, int32_t* status_word,
                               cudaStream_t st);

@@ -1,8 +1,9 @@
 // Full causal prefill attention (Eq. 3 + causal mask, layers l < k) on the Blackwell tensor cores.
 // bf16 Q/K/V, head_dim 128, fp32 logits / softmax / accumulation, bf16 output.
 //
-// Work item = 128 query rows of NT query heads that share a kv head (NT = 2 when the GQA group size is
-// even, else 1): NT "M-tiles" with the same rows and the same key range, so they share every K/V tile.
+// Work item = two "M-tiles" of 128 query rows that share every K/V tile: two query heads of one kv group on the
+// same rows (even GQA group size), or two consecutive query tiles of one head (odd group size, multi-head
+// attention; the first tile sits out the last key tile, which lies wholly past its diagonal).
 // A small planning kernel lists the (sequence, query tile) pairs of the batch, longest key range first;
 // the main kernel is persistent (one CTA per SM) and CTA c takes items c, c + gridDim, ... of that list,
 // so every SM gets the same mix of long and short items and the pipeline below never drains between items.
@@ -40,9 +41,10 @@ constexpr int TILE = BM * HD * 2;   // bytes of one 128 x 128 bf16 tile
 constexpr int HALF = TILE / 2;      // one 64-column block of it (128 rows x 128 B)
 constexpr long long WAIT_LIMIT = 2000000000LL;     // about one second of SM clocks
 
-template <int NT>
+constexpr int NT = 2;   // M-tiles per work item
+
 struct Cfg {
-  static constexpr int NSTAGE = NT == 1 ? 6 : 5;            // ring entries (K and V tiles alternate)
+  static constexpr int NSTAGE = 5;                          // ring entries (K and V tiles alternate)
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_RING = OFF_Q + NT * TILE;
   static constexpr int OFF_BAR = OFF_RING + NSTAGE * TILE;
@@ -61,23 +63,41 @@ struct TcParams {
   float* lse;
   const int4* plan;        // one entry per (sequence, query tile): {first global row, rows of the sequence from there, tile index, sequence}
   int32_t* status;
-  int Hq, g, total, n_items, n_hp;   // n_hp = Hq / NT work items per plan entry
+  int Hq, g, total, n_items, n_hp;   // n_hp work items per plan entry
   float scale_log2;
 };
 
 struct Item {
-  int row0;      // global row of the first query of the tile
-  int rows;      // rows of the sequence from there on (>= 1); the tile holds min(rows, 128) valid rows
-  int n_tiles;   // key tiles 0 .. diagonal
   int key0;      // global row of the sequence's first key
-  int h0;        // first query head
+  int n_tiles;   // key tiles both M-tiles are run over: 0 .. the later diagonal
+  int kvh;       // kv head
+  int row0[NT];  // global row of the first query of M-tile x
+  int rows[NT];  // rows of the sequence from there on; the tile holds min(rows, 128) valid rows (none if <= 0)
+  int head[NT];  // query head of M-tile x
+  int diag[NT];  // key tile that holds M-tile x's diagonal; later tiles are invisible to it
 };
 
-__device__ __forceinline__ Item load_item(const TcParams& p, int i, int NT) {
+// Plan entry {first global row, rows of the sequence from there, level, sequence} -> work item i.
+//   two heads of a group (even group size): level = query tile; both M-tiles have the same rows and the same diagonal;
+//   two query tiles of one head (odd group size, multi-head attention): level = pair of query tiles; the first
+//   M-tile's diagonal is one key tile earlier, and it sits out the last key tile (all of it is masked for it).
+template <bool PAIR_TILES>   // false: the two M-tiles are two heads of a kv group; true: two consecutive query tiles of one head
+__device__ __forceinline__ Item load_item(const TcParams& p, int i) {
   const int e = i / p.n_hp, hp = i - e * p.n_hp;
   const int4 t = __ldg(p.plan + e);
   Item it;
-  it.row0 = t.x; it.rows = t.y; it.n_tiles = t.z + 1; it.key0 = t.x - t.z * BM; it.h0 = hp * NT;
+  if (!PAIR_TILES) {
+    it.key0 = t.x - t.z * BM;
+    it.n_tiles = t.z + 1;
+#pragma unroll
+    for (int x = 0; x < NT; ++x) { it.row0[x] = t.x; it.rows[x] = t.y; it.head[x] = hp * NT + x; it.diag[x] = t.z; }
+  } else {
+    it.key0 = t.x - t.z * (NT * BM);
+    it.n_tiles = NT * t.z + NT;
+#pragma unroll
+    for (int x = 0; x < NT; ++x) { it.row0[x] = t.x + x * BM; it.rows[x] = t.y - x * BM; it.head[x] = hp; it.diag[x] = NT * t.z + x; }
+  }
+  it.kvh = it.head[0] / p.g;
   return it;
 }
 
@@ -97,11 +117,11 @@ __device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
       "mov.b64 {%0, %1}, rd;\n\t}"
       : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
 }
-template <int NT>
-__global__ void __launch_bounds__(Cfg<NT>::THREADS, 1)
+template <bool PAIR_TILES>
+__global__ void __launch_bounds__(Cfg::THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, TcParams p) {
-  using C = Cfg<NT>;
+  using C = Cfg;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;    // swizzled tiles need 1024-byte alignment
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
@@ -149,8 +169,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       int e = 0;   // ring entries issued so far, over all items
       bool ok = true;
       for (int i = first; i < p.n_items && ok; i += stride) {
-        const Item it = load_item(p, i, NT);
-        const int kvh = it.h0 / p.g;
+        const Item it = load_item<PAIR_TILES>(p, i);
+        const int kvh = it.kvh;
         for (int t = 0; t < 2 * it.n_tiles; ++t, ++e) {
           const int st = e % C::NSTAGE;
           if (e >= C::NSTAGE &&
@@ -177,15 +197,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       int n = 0;   // items loaded so far
       bool ok = true;
       for (int i = first; i < p.n_items && ok; i += stride, ++n) {
-        const Item it = load_item(p, i, NT);
+        const Item it = load_item<PAIR_TILES>(p, i);
         for (int x = 0; x < NT; ++x) {
           if (n > 0 && !mbar_wait_bounded(bar(C::BAR_QFREE + x), (n - 1) & 1, abort_flag, WAIT_LIMIT)) {
             ok = false;
             break;
           }
           mbar_expect_tx(bar(C::BAR_QFULL + x), TILE);
-          tma_load_3d(sQ + x * TILE, &map_q, bar(C::BAR_QFULL + x), 0, it.h0 + x, it.row0);
-          tma_load_3d(sQ + x * TILE + HALF, &map_q, bar(C::BAR_QFULL + x), 64, it.h0 + x, it.row0);
+          tma_load_3d(sQ + x * TILE, &map_q, bar(C::BAR_QFULL + x), 0, it.head[x], it.row0[x]);
+          tma_load_3d(sQ + x * TILE + HALF, &map_q, bar(C::BAR_QFULL + x), 64, it.head[x], it.row0[x]);
         }
       }
       if (*abort_flag && n > 0) {
@@ -239,7 +259,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       bool ok = first < p.n_items;
       Item cur{};
       if (ok) {
-        cur = load_item(p, first, NT);
+        cur = load_item<PAIR_TILES>(p, first);
         for (int x = 0; x < NT && ok; ++x) {
           ok = wait(C::BAR_QFULL + x, 0) && (x > 0 || wait_full(0));
           if (!ok) break;
@@ -250,7 +270,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       for (int i = first; i < p.n_items && ok; i += stride, ++n_item) {
         const bool has_next = i + stride < p.n_items;
         Item nxt{};
-        if (has_next) nxt = load_item(p, i + stride, NT);
+        if (has_next) nxt = load_item<PAIR_TILES>(p, i + stride);
         const int n = cur.n_tiles;
         for (int j = 0; j < n && ok; ++j) {
           for (int x = 0; x < NT && ok; ++x) {
@@ -298,15 +318,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     int n_s = 0, n_item = 0;
     bool ok = true;
     for (int i = first; i < p.n_items && ok; i += stride, ++n_item) {
-      const Item it = load_item(p, i, NT);
-      const int h = it.h0 + x;
+      const Item it = load_item<PAIR_TILES>(p, i);
+      // this M-tile's share of the item, in registers (x is not a compile-time index)
+      const int h = x ? it.head[1] : it.head[0], my_diag = x ? it.diag[1] : it.diag[0];
+      const int my_row0 = x ? it.row0[1] : it.row0[0], my_rows = x ? it.rows[1] : it.rows[0];
       float m_ref = 0.f, l0 = 0.f, l1 = 0.f;
       for (int j = 0; j < it.n_tiles; ++j, ++n_s) {
         ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_S + x), n_s & 1, abort_flag, WAIT_LIMIT));   // warp-uniform
         if (!ok) break;
         tc_fence_after();
-        const bool diag = j == it.n_tiles - 1;        // key column c of this tile is visible to row r iff c <= r
-        const int n_chunks = diag ? wq + 1 : 4;       // 32-column chunks with a visible key for this warp's rows
+        const bool diag = j == my_diag;               // key column c of this tile is visible to row r iff c <= r
+        // 32-column chunks with a visible key for this warp's rows (none in a tile past the diagonal)
+        const int n_chunks = diag ? wq + 1 : (!PAIR_TILES || j < my_diag) ? 4 : 0;
         uint32_t a[32], b[32], pk[4][16];
         // row maximum of the visible part of S_x(j), scaled into the log2 domain (a pass of its own over TMEM)
         auto row_max = [&]() {
@@ -413,8 +436,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       tc_fence_after();
       const float l = l0 + l1;
       const float inv = 1.f / l;
-      const bool valid = row < it.rows;
-      __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) + ((int64_t)(it.row0 + row) * p.Hq + h) * HD;
+      const bool valid = row < my_rows;
+      __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) + ((int64_t)(my_row0 + row) * p.Hq + h) * HD;
       uint32_t a[32], b[32];
       tmem_ld_32x32(t_o, a);
       tmem_wait_ld(a);
@@ -436,7 +459,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         }
         if (q + 1 < 4) tmem_wait_ld(nxt);
       }
-      if (valid && p.lse != nullptr) p.lse[(int64_t)h * p.total + it.row0 + row] = (m_ref + log2f(l)) * kLn2;
+      if (valid && p.lse != nullptr) p.lse[(int64_t)h * p.total + my_row0 + row] = (m_ref + log2f(l)) * kLn2;
       tc_fence_before();   // the next item's first P V overwrites O_x; it is issued after this warp's next arrive on P_x
     }
   }
@@ -451,14 +474,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 }
 
 // ------------------------------------------------------------------------------------------------
-// planning kernel: one entry per (sequence, query tile), tiles with the longest key range first
+// planning kernel: one entry per (sequence, block of `rows` query rows), blocks with the longest key range first
+// (rows = 128: one query tile; rows = 256: a pair of query tiles)
 // ------------------------------------------------------------------------------------------------
 constexpr int PLAN_THREADS = 1024;
 constexpr int PLAN_MAX_LEVELS = 2048;   // query tiles per sequence the planner can order (256 K tokens)
 
 __global__ void __launch_bounds__(PLAN_THREADS) prefill_plan_kernel(const int32_t* cu_seqlens, int batch, int max_tiles,
-                                                                    int4* plan) {
-  // level t holds every sequence with more than t query tiles; levels are laid out from the highest down
+                                                                    int rows, int4* plan) {
+  // level t holds every sequence with more than t blocks; levels are laid out from the highest down
   __shared__ int cnt[PLAN_MAX_LEVELS];      // sequences per level, then the level's cursor
   __shared__ int off[PLAN_MAX_LEVELS];      // first entry of the level
   pdl_launch_dependents();
@@ -466,7 +490,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) prefill_plan_kernel(const int32_
   for (int t = threadIdx.x; t < max_tiles; t += PLAN_THREADS) cnt[t] = 0;
   __syncthreads();
   for (int b = threadIdx.x; b < batch; b += PLAN_THREADS) {
-    const int n = (cu_seqlens[b + 1] - cu_seqlens[b] + BM - 1) / BM;
+    const int n = (cu_seqlens[b + 1] - cu_seqlens[b] + rows - 1) / rows;
     if (n > 0) atomicAdd(&cnt[min(n, max_tiles) - 1], 1);   // histogram by tile count first
   }
   __syncthreads();
@@ -482,8 +506,8 @@ __global__ void __launch_bounds__(PLAN_THREADS) prefill_plan_kernel(const int32_
   __syncthreads();
   for (int b = threadIdx.x; b < batch; b += PLAN_THREADS) {
     const int lo = cu_seqlens[b], len = cu_seqlens[b + 1] - lo;
-    const int n = min((len + BM - 1) / BM, max_tiles);
-    for (int t = 0; t < n; ++t) plan[off[t] + atomicAdd(&cnt[t], 1)] = make_int4(lo + t * BM, len - t * BM, t, b);
+    const int n = min((len + rows - 1) / rows, max_tiles);
+    for (int t = 0; t < n; ++t) plan[off[t] + atomicAdd(&cnt[t], 1)] = make_int4(lo + t * rows, len - t * rows, t, b);
   }
 }
 
@@ -525,23 +549,16 @@ int sm_count() {
   return n;
 }
 
-template <int NT>
-cudaError_t launch_nt(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, TcParams p, cudaStream_t st) {
-  cudaError_t e = ensure_dynamic_smem<prefill_tc_kernel<NT>>(Cfg<NT>::SMEM_BYTES);
-  if (e != cudaSuccess) return e;
-  p.n_hp = p.Hq / NT;
-  p.n_items *= p.n_hp;
-  const int grid = p.n_items < sm_count() ? p.n_items : sm_count();
-  e = launch_pdl(prefill_tc_kernel<NT>, dim3(grid), dim3(Cfg<NT>::THREADS), Cfg<NT>::SMEM_BYTES, st, mq, mk, mv, p);
-  note_launch();
-  return e != cudaSuccess ? e : cudaGetLastError();
-}
-
 }  // namespace
 
-int prefill_plan_entries(const earn_batch_t& b) {
+int prefill_rows_per_entry(int n_q_heads, int n_kv_heads) {
+  // an even group: the two M-tiles of an item are two heads on the same 128 rows; otherwise two consecutive query tiles
+  return (n_q_heads / n_kv_heads) % 2 == 0 ? BM : NT * BM;
+}
+
+int prefill_plan_entries(const earn_batch_t& b, int rows) {
   int64_t n = 0;
-  for (int i = 0; i < b.batch; ++i) n += (b.cu_seqlens_host[i + 1] - b.cu_seqlens_host[i] + BM - 1) / BM;
+  for (int i = 0; i < b.batch; ++i) n += (b.cu_seqlens_host[i + 1] - b.cu_seqlens_host[i] + rows - 1) / rows;
   return n > INT32_MAX ? INT32_MAX : (int)n;
 }
 
@@ -556,17 +573,31 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int plan_e
       !make_map(&mv, a.v, a.Hkv, total_tokens))
     return cudaErrorInvalidValue;
   if (plan_entries <= 0) return cudaSuccess;
+  const int rows = prefill_rows_per_entry(a.Hq, a.Hkv);
   cudaError_t e = launch_pdl(prefill_plan_kernel, dim3(1), dim3(PLAN_THREADS), 0, st, a.cu_seqlens, a.batch,
-                             (a.max_seqlen + BM - 1) / BM, reinterpret_cast<int4*>(plan));
+                             (a.max_seqlen + rows - 1) / rows, rows, reinterpret_cast<int4*>(plan));
   note_launch();
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   TcParams p{};
   p.o = a.o; p.lse = a.lse; p.plan = reinterpret_cast<const int4*>(plan); p.status = status_word;
-  p.Hq = a.Hq; p.g = a.Hq / a.Hkv; p.total = total_tokens; p.n_items = plan_entries;
+  p.Hq = a.Hq; p.g = a.Hq / a.Hkv; p.total = total_tokens;
+  const bool pair_tiles = rows != BM;
+  p.n_hp = pair_tiles ? a.Hq : a.Hq / NT;
+  p.n_items = plan_entries * p.n_hp;
   p.scale_log2 = a.scale * kLog2e;
-  // two query heads of one kv head per work item when the group size allows it
-  return (p.g % 2 == 0) ? launch_nt<2>(mq, mk, mv, p, st) : launch_nt<1>(mq, mk, mv, p, st);
+  const int grid = p.n_items < sm_count() ? p.n_items : sm_count();
+  if (pair_tiles) {
+    e = ensure_dynamic_smem<prefill_tc_kernel<true>>(Cfg::SMEM_BYTES);
+    if (e == cudaSuccess)
+      e = launch_pdl(prefill_tc_kernel<true>, dim3(grid), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, mq, mk, mv, p);
+  } else {
+    e = ensure_dynamic_smem<prefill_tc_kernel<false>>(Cfg::SMEM_BYTES);
+    if (e == cudaSuccess)
+      e = launch_pdl(prefill_tc_kernel<false>, dim3(grid), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, mq, mk, mv, p);
+  }
+  note_launch();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace earn
