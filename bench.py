@@ -118,7 +118,7 @@ class ClockSampler:
             pass
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", ident, f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -502,10 +502,12 @@ def blas_threads() -> int:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="7b", choices=sorted(wl.CONFIGS))
     ap.add_argument("--split-k", type=int, default=None)
+    ap.add_argument("--prompt-len", type=int, default=None, help="override the workload's prompt length (uniform)")
+    ap.add_argument("--batch", type=int, default=None, help="override the workload's batch size")
     ap.add_argument("--impl", default="earn", choices=["earn", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -526,6 +528,10 @@ def main():
     w = wl.CONFIGS[args.config]
     if args.split_k is not None:
         w = w.replace(split_k=args.split_k)
+    if args.prompt_len is not None:
+        w = w.replace(prompt_len=args.prompt_len, lens=())
+    if args.batch is not None:
+        w = w.replace(batch=args.batch)
     lens = wl.seqlens(w)
     tokens_per_step = int(lens.sum()) + w.batch * w.beams * w.decode_steps
     config = {"workload": workload_desc(w), "l2": "per-layer inputs and caches exceed the 126 MB L2; no flush needed",

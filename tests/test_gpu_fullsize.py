@@ -117,3 +117,9 @@ def test_fullsize_long_history():
 
 def test_fullsize_ragged_beams():
     run_fullsize(wl.CONFIGS["ragged"], decode_steps=3, n_random=800, n_decode_rows=300)
+
+
+def test_long_context_20k_tokens():
+    # the paper pads prompts up to 20K tokens for its length study (Section 4, sequence-length scaling): 160 key
+    # tiles per query tile in prefill, split-KV decode over a 20K-token prompt cache
+    run_fullsize(wl.CONFIGS["long"].replace(name="20k", batch=2, prompt_len=20480, seed=6), n_random=500, n_decode_rows=150)
