@@ -368,7 +368,12 @@ class GpuJob:
 # the CPU oracle arm (a baseline, not a target): one sequence of the workload through every layer and step
 # ------------------------------------------------------------------------------------------------
 class OracleSample:
-    def __init__(self, w: wl.Workload, job: GpuJob | None):
+    def __init__(self, w: wl.Workload, job: GpuJob | None, layer_stride: int = 1):
+        """One sequence of the workload through every `layer_stride`-th layer (all decode steps); with a stride the
+        measured time is scaled back by it, which keeps the full/register layer mix when the stride divides k and N."""
+        if layer_stride > 1 and (w.split_k % layer_stride or w.n_layers % layer_stride):
+            layer_stride = 1
+        self.stride = layer_stride
         lens = wl.seqlens(w)
         cu = wl.cu_seqlens(w)
         self.w1 = w.replace(batch=1, lens=(int(lens[0]),))
@@ -378,13 +383,16 @@ class OracleSample:
             self.dec = [[tuple(f(t[:w.beams]) for t in trip) for trip in row] for row in job.dec]
         else:                     # no device: draw the one-sequence workload on the host
             dev = "cuda" if torch.cuda.is_available() else "cpu"
-            self.qkv = [tuple(f(t) for t in wl.layer_qkv(self.w1, l, dev)) for l in range(w.n_layers)]
-            self.dec = [[tuple(f(t) for t in wl.decode_qkv(self.w1, l, s, dev)) for l in range(w.n_layers)]
+            every = lambda l, fn: fn() if l % layer_stride == 0 else None   # noqa: E731
+            self.qkv = [every(l, lambda: tuple(f(t) for t in wl.layer_qkv(self.w1, l, dev))) for l in range(w.n_layers)]
+            self.dec = [[every(l, lambda: tuple(f(t) for t in wl.decode_qkv(self.w1, l, s, dev))) for l in range(w.n_layers)]
                         for s in range(1, w.decode_steps + 1)]
         self.parents = [None] + [wl.beam_parents(w, s)[:w.beams] if w.beams > 1 else None
                                  for s in range(2, w.decode_steps + 1)]
         self.tokens = int(lens[0]) + w.beams * w.decode_steps
-        self.desc = (f"sequence 0 of {w.batch} (L={int(lens[0])}, {w.beams} beam(s)): all {w.n_layers} layers of prefill "
+        layers = f"all {w.n_layers} layers" if layer_stride == 1 else \
+            f"every {layer_stride}th of the {w.n_layers} layers (time scaled by {layer_stride})"
+        self.desc = (f"sequence 0 of {w.batch} (L={int(lens[0])}, {w.beams} beam(s)): {layers} of prefill "
                      f"and all {w.decode_steps} decode steps")
 
     def run(self) -> float:
@@ -393,21 +401,22 @@ class OracleSample:
         t0 = time.perf_counter()
         cu = np.array([0, w.lens[0]])
         idx = orc.register_indices(w.lens, w.r_head, w.r_tail)
-        states = []
-        for layer in range(w.n_layers):
+        states = {}
+        layers = range(0, w.n_layers, self.stride)
+        for layer in layers:
             q, k, v = self.qkv[layer]
             if layer < w.split_k:
                 orc.causal_attention(q, k, v, cu)
-                states.append(orc.DecodeState([k], [v], w.beams))
+                states[layer] = orc.DecodeState([k], [v], w.beams)
             else:
                 kc, vc, qc = orc.compact(k, cu, idx), orc.compact(v, cu, idx), orc.compact(q, cu, idx)
                 orc.register_attention(qc, kc, vc)
-                states.append(orc.DecodeState([kc[0]], [vc[0]], w.beams))
+                states[layer] = orc.DecodeState([kc[0]], [vc[0]], w.beams)
         for s in range(1, w.decode_steps + 1):
-            for layer in range(w.n_layers):
+            for layer in layers:
                 q, k, v = self.dec[s - 1][layer]
                 states[layer].step(q, k, v, self.parents[s - 1])
-        return time.perf_counter() - t0
+        return (time.perf_counter() - t0) * self.stride
 
 
 def profile_one_kernel(w: wl.Workload, dev, which: str, launches: int = 3):
@@ -540,7 +549,7 @@ def main():
     if args.impl == "reference":
         if rank != 0:
             return
-        sample = OracleSample(w, None)
+        sample = OracleSample(w, None, layer_stride=4)   # about a second of oracle work per step
         for _ in range(args.warmup):
             sample.run()
         times = [sample.run() for _ in range(args.steps)]

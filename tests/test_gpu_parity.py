@@ -154,3 +154,10 @@ def test_prefill_logits_that_keep_rising_take_the_rescale_path():
     o = make_session(w).prefill_layer(0, q, k, v)
     ref, _ = orc.causal_attention(to_np(q), to_np(k), to_np(v), cu)
     assert_close(o, ref, "bf16", "prefill with rising logits")
+
+
+def test_one_token_sequences_among_long_ones():
+    """Sequences of one and two tokens packed between long ones: the plan of the tensor-core prefill gets entries
+    of a single valid row, compaction keeps the only token, decode sees a one-key prompt cache."""
+    run_workload_and_compare(BASE.replace(seed=29, lens=(1, 300, 2, 129, 1), batch=5, r_head=1, r_tail=0, beams=2,
+                                          decode_steps=2))
