@@ -80,6 +80,16 @@ CONFIGS: Dict[str, Workload] = {
                        dtype="bf16", prompt_len=0, len_lo=128, len_hi=2048, r_head=16, r_tail=16,
                        decode_steps=20, beams=10, seed=5),
 }
+# The operating points of the paper's own measurements (Section 4 and Appendix A.3: prompts of 50-200 tokens, one
+# register per side, beam 20, item identifiers of 4 tokens, split k = 4 on the multi-head backbone at batch 24 and
+# k = 7 on the grouped-query backbone at batch 48), as shapes only.  They are extra workloads for tests and
+# timing; the benchmark's headline stays the 7B-class configuration.
+CONFIGS["paper_mha"] = Workload("paper_mha", batch=24, n_layers=32, split_k=4, n_q_heads=32, n_kv_heads=32, head_dim=128,
+                                dtype="bf16", prompt_len=0, len_lo=50, len_hi=200, r_head=1, r_tail=1, decode_steps=4,
+                                beams=20, seed=6)
+CONFIGS["paper_gqa"] = Workload("paper_gqa", batch=48, n_layers=28, split_k=7, n_q_heads=28, n_kv_heads=4, head_dim=128,
+                                dtype="bf16", prompt_len=0, len_lo=50, len_hi=200, r_head=1, r_tail=1, decode_steps=4,
+                                beams=20, seed=7)
 LONG_SPLIT_SWEEP = (2, 4, 8, 16)
 
 _TAG = {"q": 1, "k": 2, "v": 3, "dq": 4, "dk": 5, "dv": 6, "len": 7, "u": 8, "parent": 9}

@@ -123,3 +123,12 @@ def test_long_context_20k_tokens():
     # the paper pads prompts up to 20K tokens for its length study (Section 4, sequence-length scaling): 160 key
     # tiles per query tile in prefill, split-KV decode over a 20K-token prompt cache
     run_fullsize(wl.CONFIGS["long"].replace(name="20k", batch=2, prompt_len=20480, seed=6), n_random=500, n_decode_rows=150)
+
+
+@pytest.mark.parametrize("name", ["paper_mha", "paper_gqa"])
+def test_paper_operating_points(name):
+    """The shapes the paper itself measures on: 50-200 token prompts, one register per side, beam 20, 4-token item
+    identifiers; multi-head attention (two query tiles of a head per work item, 20 query rows per kv head) and a
+    group of 7 (140 query rows per kv head: nine row tiles in three CTAs).  Every element is compared."""
+    from parity_util import run_workload_and_compare
+    run_workload_and_compare(wl.CONFIGS[name].replace(n_layers=2, split_k=1), check_lse=False)
