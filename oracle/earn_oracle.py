@@ -19,6 +19,9 @@ What pins each function (see tests/test_oracle_pins.py):
   DecodeState / decode_attention : step s equals the last row of a causal prefill
                           over prompt ++ generated; W beams equal W independent runs
   kv_entries, gamma_cache, gamma_attn, speedup : the worked example of Section 3.3
+  rms_norm, apply_rope, register_qkv : closed forms (constant rows, zero angle, norm preservation), the
+                          relative-position property of the rotation, a library rms_norm / linear call, and
+                          "project every row then gather" = "gather then project" (Eq. 2 acts per token)
 Attention values have no printed worked example in the paper, so beyond those
 pins they are parity unpinned.
 """
@@ -181,6 +184,56 @@ def register_attention_masked(q, k, v, cu_seqlens, idx: np.ndarray, scale: Optio
                 p = np.exp(row - np.max(row))
                 out[b, m, h] = (p @ v[lo:hi, h // g, :]) / np.sum(p)
     return out
+
+
+# --------------------------------------------------------------------------
+# Section 3.2, inference, register-focused process, as the paper states it: the HIDDEN STATE entering
+# layer k is cut down to the register rows, X -> X' = [X_prefix; X_suffix], and only those rows go through
+# the layer.  Eq. 2 (Q = X W_Q, K = X W_K, V = X W_V) applied to the gathered rows, inside a pre-norm
+# decoder layer with rotary position embedding; the registers keep their original positions.
+# --------------------------------------------------------------------------
+def rms_norm(x: np.ndarray, weight: np.ndarray, eps: float) -> np.ndarray:
+    """y = x / sqrt(mean(x^2) + eps) * weight over the last axis, float64."""
+    x = np.asarray(x, dtype=np.float64)
+    return x / np.sqrt(np.mean(x * x, axis=-1, keepdims=True) + eps) * np.asarray(weight, dtype=np.float64)
+
+
+def rope_tables(max_pos: int, head_dim: int, theta: float = 10000.0) -> Tuple[np.ndarray, np.ndarray]:
+    """cos / sin of pos * theta^(-2i/D), i < D/2: float64 [max_pos, D/2]."""
+    inv = theta ** (-np.arange(0, head_dim, 2, dtype=np.float64) / head_dim)
+    ang = np.arange(max_pos, dtype=np.float64)[:, None] * inv[None, :]
+    return np.cos(ang), np.sin(ang)
+
+
+def apply_rope(v: np.ndarray, cos: np.ndarray, sin: np.ndarray) -> np.ndarray:
+    """Rotate the pairs (i, i + D/2) of v [..., D] by the angles whose cos / sin are given as [..., D/2]."""
+    v = np.asarray(v, dtype=np.float64)
+    half = v.shape[-1] // 2
+    a, b = v[..., :half], v[..., half:]
+    return np.concatenate([a * cos - b * sin, b * cos + a * sin], axis=-1)
+
+
+def register_qkv(x, cu_seqlens, idx: np.ndarray, w_norm, w_qkv, n_q_heads: int, n_kv_heads: int, head_dim: int,
+                 rope_cos, rope_sin, eps: float = 1e-6):
+    """Hidden states x [total, d_model] -> (Q' [B,R,Hq,D], K' [B,R,Hkv,D], V' [B,R,Hkv,D]) of the register rows only:
+    gather rows idx[b] of every sequence, RMS-normalise, multiply by W_qkv^T (w_qkv [(Hq+2Hkv)*D, d_model], rows
+    ordered Q heads, K heads, V heads), rotate Q and K by the ORIGINAL position idx[b][m] of each register."""
+    x = np.asarray(x, dtype=np.float64)
+    w = np.asarray(w_qkv, dtype=np.float64)
+    b_, r_ = idx.shape
+    q = np.zeros((b_, r_, n_q_heads, head_dim))
+    k = np.zeros((b_, r_, n_kv_heads, head_dim))
+    v = np.zeros((b_, r_, n_kv_heads, head_dim))
+    for b in range(b_):
+        for m in range(r_):
+            pos = int(idx[b, m])
+            y = rms_norm(x[int(cu_seqlens[b]) + pos], w_norm, eps) @ w.T
+            qh = y[: n_q_heads * head_dim].reshape(n_q_heads, head_dim)
+            kh = y[n_q_heads * head_dim:(n_q_heads + n_kv_heads) * head_dim].reshape(n_kv_heads, head_dim)
+            q[b, m] = apply_rope(qh, rope_cos[pos], rope_sin[pos])
+            k[b, m] = apply_rope(kh, rope_cos[pos], rope_sin[pos])
+            v[b, m] = y[(n_q_heads + n_kv_heads) * head_dim:].reshape(n_kv_heads, head_dim)
+    return q, k, v
 
 
 # --------------------------------------------------------------------------

@@ -332,3 +332,52 @@ def test_synthetic_inputs_show_dual_sinks():
         tails.append(b)
     # 2 sink keys of weight ~e^4 among 256 ordinary ones: each side holds a visible share
     assert np.mean(heads) > 0.08 and np.mean(tails) > 0.08
+
+
+# ---- the hidden-state form of the register-focused process (gather X -> X', then Eq. 2 on the register rows)
+def test_rms_norm_and_rope_closed_forms():
+    x = np.full((3, 8), 2.0)
+    assert np.allclose(orc.rms_norm(x, np.arange(8.0), 0.0), np.tile(np.arange(8.0), (3, 1)))     # x / |x|_rms = 1
+    cos, sin = orc.rope_tables(16, 8)
+    v = np.random.default_rng(0).standard_normal((5, 8))
+    assert np.allclose(orc.apply_rope(v, cos[0], sin[0]), v)                                       # position 0: identity
+    for pos in (1, 7, 15):
+        assert np.allclose(np.linalg.norm(orc.apply_rope(v, cos[pos], sin[pos]), axis=-1), np.linalg.norm(v, axis=-1))
+    # the score of a rotated query and key depends on the distance between their positions only
+    q, k = v[0], v[1]
+    s1 = orc.apply_rope(q, cos[9], sin[9]) @ orc.apply_rope(k, cos[4], sin[4])
+    s2 = orc.apply_rope(q, cos[14], sin[14]) @ orc.apply_rope(k, cos[9], sin[9])
+    assert np.isclose(s1, s2)
+    # lowest pair at position p is a plane rotation by p radians (theta^0 = 1)
+    r = orc.apply_rope(np.array([1.0, 0, 0, 0, 0.0, 0, 0, 0]), cos[3], sin[3])
+    assert np.allclose([r[0], r[4]], [np.cos(3.0), np.sin(3.0)])
+
+
+def test_register_qkv_matches_library_ops_and_commutes_with_the_gather():
+    rng = np.random.default_rng(5)
+    lens, rh, rt, dm, hq, hkv, d = (9, 6), 2, 1, 32, 4, 2, 8
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    x = rng.standard_normal((cu[-1], dm))
+    wn = rng.standard_normal(dm)
+    w = rng.standard_normal(((hq + 2 * hkv) * d, dm)) / np.sqrt(dm)
+    cos, sin = orc.rope_tables(16, d)
+    idx = orc.register_indices(lens, rh, rt)
+    q, k, v = orc.register_qkv(x, cu, idx, wn, w, hq, hkv, d, cos, sin, eps=1e-6)
+    # library: normalise and project EVERY token, rotate by its own position, then gather the register rows
+    xt = torch.from_numpy(x)
+    y = torch.nn.functional.linear(torch.nn.functional.rms_norm(xt, (dm,), torch.from_numpy(wn), 1e-6), torch.from_numpy(w)).numpy()
+    for b in range(2):
+        for m in range(rh + rt):
+            pos = idx[b, m]
+            row = y[cu[b] + pos]
+            assert np.allclose(q[b, m], orc.apply_rope(row[:hq * d].reshape(hq, d), cos[pos], sin[pos]))
+            assert np.allclose(k[b, m], orc.apply_rope(row[hq * d:(hq + hkv) * d].reshape(hkv, d), cos[pos], sin[pos]))
+            assert np.allclose(v[b, m], row[(hq + hkv) * d:].reshape(hkv, d))
+    # rows outside the registers do not matter
+    x2 = x.copy()
+    keep = np.zeros(cu[-1], bool)
+    for b in range(2):
+        keep[cu[b] + idx[b]] = True
+    x2[~keep] = rng.standard_normal((int((~keep).sum()), dm))
+    q2, k2, v2 = orc.register_qkv(x2, cu, idx, wn, w, hq, hkv, d, cos, sin, eps=1e-6)
+    assert np.array_equal(q, q2) and np.array_equal(k, k2) and np.array_equal(v, v2)
