@@ -94,6 +94,9 @@ def algorithmic(w: wl.Workload):
                           bytes=float(tot * D * es * (2 * Hq + 2 * Hkv)))
     out["compact"] = dict(flops=0.0, bytes=float(2 * B * R * D * es * (2 * Hkv + Hq) + B * R * 4))
     out["register"] = dict(flops=4.0 * D * Hq * B * R * (R + 1) / 2, bytes=float(B * R * D * es * (2 * Hq + 2 * Hkv)))
+    # hidden-state form of a register layer: the projection of the B*R register rows (bf16 path only)
+    M, N, K = B * R, (Hq + 2 * Hkv) * D, w.d_model
+    out["register_qkv"] = dict(flops=2.0 * M * N * K, bytes=float(es * (3 * M * K + N * K + M * N + K)))
     s = w.decode_steps   # last step: the longest cache
     qo = 2 * B * W * Hq * D * es + 4 * B * W * Hkv * D * es
     out["decode_compact"] = dict(flops=4.0 * D * Hq * B * W * (R + s), bytes=float(2 * B * (R + W * s) * Hkv * D * es + qo))
@@ -281,6 +284,17 @@ class GpuJob:
                                                                    caches[l], self.qkv[l][0], self.q_reg) for l in late], len(late))
             res["register"] = timed(lambda: [self.B.earn_register_attn(ses.model, ses.batch, l, self.q_reg, caches[l],
                                                                        self.o_reg, ses.workspace) for l in late], len(late))
+            if w.dtype == "bf16" and w.head_dim == 128 and w.n_regs > 0:
+                # the same layers from hidden states (not part of the timed step, whose inputs are Q, K, V): one x for
+                # every layer, weights per layer so that they come from HBM as they would in a model
+                ses.set_projection(w.d_model, int(wl.seqlens(w).max()))
+                x = wl.hidden_states(w, late[0], self.dev)
+                wts = [wl.projection_weights(w, l, self.dev) for l in late]
+                proj = self.B.make_proj(w.d_model, ses.rope_cos, ses.rope_sin)
+                res["register_qkv"] = timed(lambda: [self.B.earn_register_qkv(ses.model, ses.batch, l, proj, x, wts[i][0], wts[i][1],
+                                                                              ses.x_norm, caches[l], self.q_reg, ses.workspace)
+                                                     for i, l in enumerate(late)], len(late))
+                del x, wts
         if w.decode_steps > 0:
             s = w.decode_steps
             if late:

@@ -8,6 +8,7 @@
  *
  *   layers l <  k : earn_prefill_attn                       (prefill)   earn_decode_attn with k_full/v_full (decode)
  *   layers l >= k : earn_compact_kv -> earn_register_attn    (prefill)   earn_decode_attn over the compact cache (decode)
+ *                   (or earn_register_qkv -> earn_register_attn when the caller hands over hidden states and W_qkv)
  *
  * Layers are 0-indexed: 0..k-1 are full layers, k..N-1 register layers.
  *
@@ -131,6 +132,32 @@ earn_status_t earn_prefill_attn(const earn_model_t* model, const earn_batch_t* b
 earn_status_t earn_compact_kv(const earn_model_t* model, const earn_batch_t* batch, int32_t layer,
                               const void* k, const void* v, const void* q_or_null, void* q_reg_or_null,
                               const earn_cache_t* cache, earn_stream_t stream);
+
+/* Projection of a layer l >= k from the hidden states (the paper's own statement of the register-focused process). */
+typedef struct {
+  int32_t d_model;        /* hidden size; a multiple of 64 */
+  int32_t max_pos;        /* rows of the rotary tables; every prompt position must be below it */
+  float   rms_eps;        /* epsilon of the RMS normalisation */
+  int32_t x_is_compact;   /* 0: x holds every prompt token, [total_tokens, d_model];
+                             1: x holds the register rows only, [B*R, d_model] (layers after the first register layer) */
+  const float* rope_cos;  /* device fp32 [max_pos, D/2]: cos(pos * theta^(-2i/D)) */
+  const float* rope_sin;  /* device fp32 [max_pos, D/2] */
+} earn_proj_t;
+
+/* Steps 2+ fused with the projection — Section 3.2 "Register-Focused Process", Eq. 2 restricted to X' = [prefix; suffix]:
+ *   X_n = RMSNorm(X'[b,m]) * w_norm;   [Q' K' V'] = X_n W_qkv^T;   Q', K' rotated by the ORIGINAL position idx_b[m]
+ * (rotary pairs (i, i + D/2)).  K', V' go to row m of sequence b's compact cache pages, Q' to q_reg (device [B, R, Hq, D]),
+ * idx to cache->reg_idx if it is not NULL: the state earn_compact_kv leaves, without K/V of the other prompt tokens ever
+ * being computed.  bf16 only, head_dim 128.
+ * x: device bf16 (see x_is_compact); w_norm: device bf16 [d_model]; w_qkv: device bf16 [(Hq+2Hkv)*D, d_model], rows in the
+ * order Q heads, K heads, V heads; x_norm_scratch: device bf16 [B*R, d_model], caller-owned, overwritten.
+ * Arithmetic: fp32 sum of squares, X_n rounded to bf16, fp32 tensor-core accumulation, fp32 rotation, one rounding to bf16.
+ * Errors: layer outside [k,N), d_model % 64 != 0, a prompt longer than max_pos -> INVALID_ARG; fp32 model or
+ * head_dim != 128 -> UNSUPPORTED; workspace NULL / too small -> WORKSPACE. */
+earn_status_t earn_register_qkv(const earn_model_t* model, const earn_batch_t* batch, int32_t layer,
+                                const earn_proj_t* proj, const void* x, const void* w_norm, const void* w_qkv,
+                                void* x_norm_scratch, const earn_cache_t* cache, void* q_reg,
+                                void* workspace, size_t workspace_bytes, earn_stream_t stream);
 
 /* Step 3 — attention of a layer l >= k during prefill: causal attention among the R register tokens of
  * each sequence in the order [prefix; suffix] (Section 3.2, training rule "only register ... tokens

@@ -42,6 +42,11 @@ class EarnCache(C.Structure):
                 ("beams", C.c_int32), ("max_new", C.c_int32), ("reg_idx", C.c_void_p)]
 
 
+class EarnProj(C.Structure):
+    _fields_ = [("d_model", C.c_int32), ("max_pos", C.c_int32), ("rms_eps", C.c_float), ("x_is_compact", C.c_int32),
+                ("rope_cos", C.c_void_p), ("rope_sin", C.c_void_p)]
+
+
 SYMBOLS = {
     "earn_workspace_bytes": (C.c_size_t, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32]),
     "earn_workspace_init": (C.c_int, [C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -51,6 +56,9 @@ SYMBOLS = {
                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "earn_compact_kv": (C.c_int, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32, C.c_void_p, C.c_void_p,
                                   C.c_void_p, C.c_void_p, C.POINTER(EarnCache), C.c_void_p]),
+    "earn_register_qkv": (C.c_int, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32, C.POINTER(EarnProj), C.c_void_p,
+                                    C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(EarnCache), C.c_void_p, C.c_void_p,
+                                    C.c_size_t, C.c_void_p]),
     "earn_register_attn": (C.c_int, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32, C.c_void_p,
                                      C.POINTER(EarnCache), C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "earn_decode_attn": (C.c_int, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32, C.c_int32, C.c_void_p,
@@ -183,6 +191,20 @@ def earn_prefill_attn(model, batch: Batch, layer, q, k, v, o, lse=None, workspac
 def earn_compact_kv(model, batch: Batch, layer, k, v, cache: EarnCache, q=None, q_reg=None) -> None:
     _check(lib().earn_compact_kv(C.byref(model), C.byref(batch.c), layer, _ptr(k), _ptr(v), _ptr(q), _ptr(q_reg),
                                  C.byref(cache), _stream()), "earn_compact_kv")
+
+
+def make_proj(d_model: int, rope_cos: torch.Tensor, rope_sin: torch.Tensor, rms_eps: float = 1e-6,
+              x_is_compact: bool = False) -> EarnProj:
+    """rope_cos / rope_sin: device fp32 [max_pos, D/2], kept alive by the caller."""
+    return EarnProj(d_model, rope_cos.shape[0], rms_eps, int(x_is_compact), _ptr(rope_cos), _ptr(rope_sin))
+
+
+def earn_register_qkv(model, batch: Batch, layer, proj: EarnProj, x, w_norm, w_qkv, x_norm_scratch, cache: EarnCache,
+                      q_reg, workspace=None) -> None:
+    p, n = _ws(workspace)
+    _check(lib().earn_register_qkv(C.byref(model), C.byref(batch.c), layer, C.byref(proj), _ptr(x), _ptr(w_norm),
+                                   _ptr(w_qkv), _ptr(x_norm_scratch), C.byref(cache), _ptr(q_reg), p, n, _stream()),
+           "earn_register_qkv")
 
 
 def earn_register_attn(model, batch: Batch, layer, q_reg, cache: EarnCache, o_reg, workspace=None) -> None:

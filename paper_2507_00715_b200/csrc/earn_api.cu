@@ -217,6 +217,39 @@ earn_status_t earn_compact_kv(const earn_model_t* model, const earn_batch_t* bat
   return launch_compact(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
 }
 
+earn_status_t earn_register_qkv(const earn_model_t* model, const earn_batch_t* batch, int32_t layer,
+                                const earn_proj_t* proj, const void* x, const void* w_norm, const void* w_qkv,
+                                void* x_norm_scratch, const earn_cache_t* cache, void* q_reg, void* workspace,
+                                size_t workspace_bytes, earn_stream_t stream) {
+  earn_status_t s = check_model(model);
+  if (s != EARN_OK) return s;
+  s = check_batch(batch);
+  if (s != EARN_OK) return s;
+  if (layer < model->split_k || layer >= model->n_layers || proj == nullptr) return EARN_ERR_INVALID_ARG;
+  if (model->dtype != EARN_BF16 || model->head_dim != 128) return EARN_ERR_UNSUPPORTED;
+  if (proj->d_model <= 0 || proj->d_model % 64 != 0 || proj->max_pos <= 0 || !(proj->rms_eps >= 0.f)) return EARN_ERR_INVALID_ARG;
+  if (batch->max_seqlen > proj->max_pos) return EARN_ERR_INVALID_ARG;
+  s = check_cache_shared(model, batch, cache);
+  if (s != EARN_OK) return s;
+  const int R = batch->n_head_reg + batch->n_tail_reg;
+  if (R == 0 || batch->batch == 0) return EARN_OK;
+  if ((int64_t)batch->batch * R > (int64_t)1 << 24) return EARN_ERR_UNSUPPORTED;
+  if (!x || !w_norm || !w_qkv || !x_norm_scratch || !q_reg || !proj->rope_cos || !proj->rope_sin) return EARN_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(w_norm) || !aligned16(w_qkv) || !aligned16(x_norm_scratch) || !aligned16(q_reg))
+    return EARN_ERR_INVALID_ARG;
+  if (workspace == nullptr || workspace_bytes < (size_t)kStatusBytes) return EARN_ERR_WORKSPACE;
+  RegisterQkvArgs a{};
+  a.x = x; a.w_norm = w_norm; a.w_qkv = w_qkv; a.x_norm = x_norm_scratch; a.q_reg = q_reg;
+  a.cache = paged_source(batch, cache);
+  a.cu_seqlens = batch->cu_seqlens; a.reg_idx = cache->reg_idx;
+  a.rope_cos = proj->rope_cos; a.rope_sin = proj->rope_sin;
+  a.status = reinterpret_cast<int32_t*>(workspace);
+  a.batch = batch->batch; a.R = R; a.r_head = batch->n_head_reg; a.r_tail = batch->n_tail_reg;
+  a.Hq = model->n_q_heads; a.Hkv = model->n_kv_heads; a.d_model = proj->d_model;
+  a.x_is_compact = proj->x_is_compact != 0; a.max_pos = proj->max_pos; a.rms_eps = proj->rms_eps;
+  return launch_register_qkv(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+}
+
 earn_status_t earn_register_attn(const earn_model_t* model, const earn_batch_t* batch, int32_t layer,
                                  const void* q_reg, const earn_cache_t* cache, void* o_reg, void* workspace,
                                  size_t workspace_bytes, earn_stream_t stream) {

@@ -153,6 +153,20 @@ struct CompactArgs {
 };
 cudaError_t launch_compact(const CompactArgs& a, cudaStream_t st);
 
+// register rows of a layer l >= k straight from the hidden states: gather, RMSNorm, QKV projection, rotary embedding
+struct RegisterQkvArgs {
+  const void *x, *w_norm, *w_qkv;
+  void *x_norm, *q_reg;
+  KeySource cache;             // paged compact cache the K and V rows are written to
+  const int32_t* cu_seqlens;
+  int32_t* reg_idx;
+  const float *rope_cos, *rope_sin;
+  int32_t* status;
+  int batch, R, r_head, r_tail, Hq, Hkv, d_model, x_is_compact, max_pos;
+  float rms_eps;
+};
+cudaError_t launch_register_qkv(const RegisterQkvArgs& a, cudaStream_t st);
+
 cudaError_t launch_beam_reparent(int batch, int beams, int max_new, int step, const int32_t* parent,
                                  const int32_t* lineage_in, int32_t* lineage_out, cudaStream_t st);
 

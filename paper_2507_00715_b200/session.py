@@ -84,6 +84,33 @@ class EarnSession:
         self.last_q_reg = q_reg
         return o
 
+    def set_projection(self, d_model: int, max_pos: int, theta: float = 10000.0, rms_eps: float = 1e-6) -> None:
+        """Rotary tables (angles pos * theta^(-2i/D), evaluated in double, stored fp32) and the scratch the
+        hidden-state form of the register layers needs."""
+        inv = theta ** (-torch.arange(0, self.D, 2, dtype=torch.float64) / self.D)
+        ang = torch.arange(max_pos, dtype=torch.float64)[:, None] * inv[None, :]
+        self.rope_cos = torch.cos(ang).float().to(self.device)
+        self.rope_sin = torch.sin(ang).float().to(self.device)
+        self.d_model, self.rms_eps = d_model, rms_eps
+        self.x_norm = torch.empty(max(self.batch.batch * self.R, 1), d_model, device=self.device, dtype=self.dtype)
+
+    def register_layer_from_hidden(self, layer: int, x: torch.Tensor, w_norm: torch.Tensor, w_qkv: torch.Tensor,
+                                   x_is_compact: bool = False, out: Optional[torch.Tensor] = None,
+                                   q_reg: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Layer >= k from the hidden states: projection of the register rows into the compact cache, then register
+        attention.  Returns O' [B,R,Hq,D]; call set_projection() first."""
+        nb = self.batch.batch
+        if q_reg is None:
+            q_reg = torch.empty(nb, self.R, self.Hq, self.D, device=self.device, dtype=self.dtype)
+        o = out if out is not None else torch.empty_like(q_reg)
+        cache = self.cache(layer)
+        proj = B.make_proj(self.d_model, self.rope_cos, self.rope_sin, self.rms_eps, x_is_compact)
+        B.earn_register_qkv(self.model, self.batch, layer, proj, x, w_norm, w_qkv, self.x_norm, cache, q_reg,
+                            self.workspace)
+        B.earn_register_attn(self.model, self.batch, layer, q_reg, cache, o, self.workspace)
+        self.last_q_reg = q_reg
+        return o
+
     # ---- decode
     def begin_step(self, step: int, parents: Optional[torch.Tensor]) -> None:
         """Re-parent the beams before decode step `step` (>= 2); parents: int32 device [B*W]."""

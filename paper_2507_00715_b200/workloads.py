@@ -17,6 +17,10 @@ Recipe, per layer and per tensor (fresh generator seeded from
   logit of every query toward the two sink keys have mean +4;
 * the result is rounded once to the workload dtype (bf16 or fp32).
 
+Hidden-state form of the register layers: X ~ N(0,1) [rows, d_model], the
+normalisation weight 1 + 0.1 N(0,1), W_qkv ~ N(0, 1/d_model), each rounded once
+to the workload dtype.
+
 Decode-step tensors (one new token per beam) are drawn the same way; beam
 parents are uniform integers in [0, W).
 """
@@ -50,6 +54,7 @@ class Workload:
     seed: int = 0
     sink_q_bias: bool = True
     lens: Tuple[int, ...] = ()   # explicit prompt lengths (tests); overrides prompt_len / len_lo / len_hi
+    hidden: int = 0        # d_model of the hidden-state form of the register layers; 0 => Hq * D
 
     @property
     def group(self) -> int:
@@ -58,6 +63,10 @@ class Workload:
     @property
     def n_regs(self) -> int:
         return self.r_head + self.r_tail
+
+    @property
+    def d_model(self) -> int:
+        return self.hidden if self.hidden > 0 else self.n_q_heads * self.head_dim
 
     @property
     def torch_dtype(self) -> torch.dtype:
@@ -92,7 +101,7 @@ CONFIGS["paper_gqa"] = Workload("paper_gqa", batch=48, n_layers=28, split_k=7, n
                                 beams=20, seed=7)
 LONG_SPLIT_SWEEP = (2, 4, 8, 16)
 
-_TAG = {"q": 1, "k": 2, "v": 3, "dq": 4, "dk": 5, "dv": 6, "len": 7, "u": 8, "parent": 9}
+_TAG = {"q": 1, "k": 2, "v": 3, "dq": 4, "dk": 5, "dv": 6, "len": 7, "u": 8, "parent": 9, "x": 10, "wn": 11, "wqkv": 12}
 
 
 def _seed_for(w: Workload, tag: str, layer: int = 0, step: int = 0) -> int:
@@ -148,6 +157,21 @@ def layer_qkv(w: Workload, layer: int, device="cpu") -> Tuple[torch.Tensor, torc
         q += math.sqrt(w.head_dim) * u.repeat_interleave(w.group, dim=0)
     dt = w.torch_dtype
     return q.to(dt), k.to(dt), v.to(dt)
+
+
+def hidden_states(w: Workload, layer: int, device="cpu", compact: bool = False) -> torch.Tensor:
+    """Hidden states entering a layer, ~ N(0,1), in the workload dtype: [total, d_model] for every prompt token, or
+    (compact) [B*R, d_model] for the register rows alone."""
+    rows = w.batch * w.n_regs if compact else int(cu_seqlens(w)[-1])
+    return _randn((rows, w.d_model), _seed_for(w, "x", layer, int(compact)), device).to(w.torch_dtype)
+
+
+def projection_weights(w: Workload, layer: int, device="cpu") -> Tuple[torch.Tensor, torch.Tensor]:
+    """(w_norm [d_model] ~ 1 + 0.1 N(0,1),  w_qkv [(Hq + 2 Hkv) * D, d_model] ~ N(0, 1/d_model)), workload dtype; the
+    rows of w_qkv are ordered Q heads, K heads, V heads."""
+    wn = 1.0 + 0.1 * _randn((w.d_model,), _seed_for(w, "wn", layer), device)
+    wq = _randn(((w.n_q_heads + 2 * w.n_kv_heads) * w.head_dim, w.d_model), _seed_for(w, "wqkv", layer), device)
+    return wn.to(w.torch_dtype), (wq / math.sqrt(w.d_model)).to(w.torch_dtype)
 
 
 def decode_qkv(w: Workload, layer: int, step: int, device="cpu"):

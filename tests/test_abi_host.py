@@ -106,6 +106,31 @@ def test_host_validation_compact_register_decode(lib):
     assert lib.earn_beam_reparent(2, 3, 4, 5, 0x1000, None, 0x2000, None) == B.EARN_ERR_INVALID_ARG
 
 
+def test_host_validation_register_qkv(lib):
+    m = B.make_model(4, 2, 8, 2, 128, "bf16")
+    b = FakeBatch([40, 50], 10, 10)
+    cache = B.make_cache(0x1000, 0x1000, None, 2, 4, 0x1000, 0x1000, None, 1, 4, None)
+
+    def proj(d_model=512, max_pos=64, eps=1e-6, cos=0x1000):
+        return B.EarnProj(d_model, max_pos, eps, 0, cos, 0x1000)
+
+    def call(layer=2, p=None, model=m, x=0x1000, ws=0x1000, scratch=0x1000):
+        p = p or proj()
+        return lib.earn_register_qkv(C.byref(model), C.byref(b.c), layer, C.byref(p), x, 0x1000, 0x1000, scratch,
+                                     C.byref(cache), 0x1000, ws, 1 << 20, None)
+
+    assert call(layer=1) == B.EARN_ERR_INVALID_ARG                       # a full layer has no register projection
+    assert call(p=proj(d_model=520)) == B.EARN_ERR_INVALID_ARG           # not a multiple of 64
+    assert call(p=proj(max_pos=49)) == B.EARN_ERR_INVALID_ARG            # a 50-token prompt needs 50 table rows
+    assert call(p=proj(eps=-1.0)) == B.EARN_ERR_INVALID_ARG
+    assert call(p=proj(cos=None)) == B.EARN_ERR_INVALID_ARG
+    assert call(x=0x1008) == B.EARN_ERR_INVALID_ARG                      # 16-byte alignment
+    assert call(scratch=None) == B.EARN_ERR_INVALID_ARG
+    assert call(ws=0) == B.EARN_ERR_WORKSPACE
+    assert call(model=B.make_model(4, 2, 8, 2, 128, "f32")) == B.EARN_ERR_UNSUPPORTED
+    assert call(model=B.make_model(4, 2, 8, 2, 64, "bf16")) == B.EARN_ERR_UNSUPPORTED
+
+
 def test_workspace_size_covers_the_decode_partials(lib):
     m = B.make_model(32, 8, 32, 8, 128, "bf16")
     b = FakeBatch([4096] * 8, 16, 16)
