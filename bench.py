@@ -455,6 +455,11 @@ def profile_one_kernel(w: wl.Workload, dev, which: str, launches: int = 3):
         ses.prefill_layer(0, q, k, v, out=o)            # also registers the prompt K/V for decode
     else:
         ses.prefill_layer(1, q, k, v, out=o_reg, q_reg=q_reg)
+    if which == "register_qkv":
+        ses.set_projection(w1.d_model, int(wl.seqlens(w1).max()))
+        x = wl.hidden_states(w1, 1, dev)
+        w_norm, w_qkv = wl.projection_weights(w1, 1, dev)
+        proj = B.make_proj(w1.d_model, ses.rope_cos, ses.rope_sin)
     torch.cuda.synchronize()
     for _ in range(launches):
         if which == "prefill":
@@ -463,6 +468,8 @@ def profile_one_kernel(w: wl.Workload, dev, which: str, launches: int = 3):
             B.earn_compact_kv(ses.model, ses.batch, 1, k, v, ses.cache(1), q, q_reg)
         elif which == "register":
             B.earn_register_attn(ses.model, ses.batch, 1, q_reg, ses.cache(1), o_reg, ses.workspace)
+        elif which == "register_qkv":
+            B.earn_register_qkv(ses.model, ses.batch, 1, proj, x, w_norm, w_qkv, ses.x_norm, ses.cache(1), q_reg, ses.workspace)
         else:
             ses.decode_layer(layer, s_last, dq, dk, dv, out=o_dec)
     torch.cuda.synchronize()
@@ -537,7 +544,7 @@ def main():
     ap.add_argument("--no-parts", action="store_true")
     ap.add_argument("--no-graphs", action="store_true", help="plain launches instead of CUDA-graph replay")
     ap.add_argument("--profile-kernel", default=None,
-                    choices=["prefill", "compact", "register", "decode_compact", "decode_full"],
+                    choices=["prefill", "compact", "register", "register_qkv", "decode_compact", "decode_full"],
                     help="small case for a profiler: allocate ONE layer of the workload and launch that step 3 times")
     ap.add_argument("--sweep-k", default=None,
                     help="comma-separated split layers k: time the workload once per k (one JSON line each, k = N is the "

@@ -235,7 +235,8 @@ earn_status_t earn_register_qkv(const earn_model_t* model, const earn_batch_t* b
   if (R == 0 || batch->batch == 0) return EARN_OK;
   if ((int64_t)batch->batch * R > (int64_t)1 << 24) return EARN_ERR_UNSUPPORTED;
   if (!x || !w_norm || !w_qkv || !x_norm_scratch || !q_reg || !proj->rope_cos || !proj->rope_sin) return EARN_ERR_INVALID_ARG;
-  if (!aligned16(x) || !aligned16(w_norm) || !aligned16(w_qkv) || !aligned16(x_norm_scratch) || !aligned16(q_reg))
+  if (!aligned16(x) || !aligned16(w_norm) || !aligned16(w_qkv) || !aligned16(x_norm_scratch) || !aligned16(q_reg) ||
+      !aligned16(proj->rope_cos) || !aligned16(proj->rope_sin))
     return EARN_ERR_INVALID_ARG;
   if (workspace == nullptr || workspace_bytes < (size_t)kStatusBytes) return EARN_ERR_WORKSPACE;
   RegisterQkvArgs a{};

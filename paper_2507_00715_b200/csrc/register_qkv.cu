@@ -206,39 +206,52 @@ register_qkv_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       const float* cs = p.rope_cos + (int64_t)pos * (HD / 2);
       const float* sn = p.rope_sin + (int64_t)pos * (HD / 2);
       const int64_t page_row = valid ? key_row(p.cache, b, m) : 0;
+      // destination row and kind of each of the tile's two heads (0..Hq-1: Q; then Hkv K heads; then Hkv V heads)
+      __nv_bfloat16* dst[BN / HD];
+      bool rotate[BN / HD];
 #pragma unroll
       for (int hh = 0; hh < BN / HD; ++hh) {
-        const int head = nt * (BN / HD) + hh;   // 0..Hq-1: Q; then Hkv K heads; then Hkv V heads
-        const uint32_t t_acc = tmem + ((uint32_t)(wq * 32) << 16) + acc * BN + hh * HD;
-        __nv_bfloat16* dst = nullptr;
-        bool rotate = false;
+        const int head = nt * (BN / HD) + hh;
+        dst[hh] = nullptr;
+        rotate[hh] = head < p.Hq + p.Hkv;
         if (valid && head < p.n_heads) {
-          if (head < p.Hq) {
-            dst = reinterpret_cast<__nv_bfloat16*>(p.q_reg) + ((int64_t)row * p.Hq + head) * HD;
-            rotate = true;
-          } else if (head < p.Hq + p.Hkv) {
-            dst = reinterpret_cast<__nv_bfloat16*>(const_cast<void*>(p.cache.k)) + (page_row * p.Hkv + (head - p.Hq)) * HD;
-            rotate = true;
-          } else {
-            dst = reinterpret_cast<__nv_bfloat16*>(const_cast<void*>(p.cache.v)) + (page_row * p.Hkv + (head - p.Hq - p.Hkv)) * HD;
+          if (head < p.Hq)
+            dst[hh] = reinterpret_cast<__nv_bfloat16*>(p.q_reg) + ((int64_t)row * p.Hq + head) * HD;
+          else if (head < p.Hq + p.Hkv)
+            dst[hh] = reinterpret_cast<__nv_bfloat16*>(const_cast<void*>(p.cache.k)) + (page_row * p.Hkv + (head - p.Hq)) * HD;
+          else
+            dst[hh] = reinterpret_cast<__nv_bfloat16*>(const_cast<void*>(p.cache.v)) + (page_row * p.Hkv + (head - p.Hq - p.Hkv)) * HD;
+        }
+      }
+      // Columns i and i + 64 of a head rotate together: chunk q (32 columns) is fetched with chunk q + 2.  The angles
+      // depend on the row and on i only, so one fetch of cos / sin serves both heads of the tile.
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        float4 c4[8], s4[8];
+        if (rotate[0]) {   // heads are ordered Q, K, V: if the first does not rotate, neither does the second
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            c4[c] = __ldg(reinterpret_cast<const float4*>(cs + q * 32) + c);
+            s4[c] = __ldg(reinterpret_cast<const float4*>(sn + q * 32) + c);
           }
         }
-        // columns i and i + 64 of a head rotate together: fetch chunk q (32 columns) with chunk q + 2
+        const float* co = reinterpret_cast<const float*>(c4);
+        const float* si = reinterpret_cast<const float*>(s4);
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
+        for (int hh = 0; hh < BN / HD; ++hh) {
+          const uint32_t t_acc = tmem + ((uint32_t)(wq * 32) << 16) + acc * BN + hh * HD;
           uint32_t lo[32], hi[32];
           tmem_ld_32x32(t_acc + q * 32, lo);
           tmem_ld_32x32(t_acc + (q + 2) * 32, hi);
           tmem_wait_ld(lo);
           tmem_wait_ld(hi);
-          if (dst != nullptr) {
-            if (rotate) {
+          if (dst[hh] != nullptr) {
+            if (rotate[hh]) {
 #pragma unroll
               for (int c = 0; c < 32; ++c) {
                 const float a = __uint_as_float(lo[c]), bb = __uint_as_float(hi[c]);
-                const float co = __ldg(cs + q * 32 + c), si = __ldg(sn + q * 32 + c);
-                lo[c] = __float_as_uint(a * co - bb * si);
-                hi[c] = __float_as_uint(bb * co + a * si);
+                lo[c] = __float_as_uint(a * co[c] - bb * si[c]);
+                hi[c] = __float_as_uint(bb * co[c] + a * si[c]);
               }
             }
 #pragma unroll
@@ -252,8 +265,8 @@ register_qkv_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
               w1.y = pack_bf16(__uint_as_float(hi[c * 8 + 2]), __uint_as_float(hi[c * 8 + 3]));
               w1.z = pack_bf16(__uint_as_float(hi[c * 8 + 4]), __uint_as_float(hi[c * 8 + 5]));
               w1.w = pack_bf16(__uint_as_float(hi[c * 8 + 6]), __uint_as_float(hi[c * 8 + 7]));
-              *reinterpret_cast<uint4*>(dst + q * 32 + c * 8) = w0;
-              *reinterpret_cast<uint4*>(dst + (q + 2) * 32 + c * 8) = w1;
+              *reinterpret_cast<uint4*>(dst[hh] + q * 32 + c * 8) = w0;
+              *reinterpret_cast<uint4*>(dst[hh] + (q + 2) * 32 + c * 8) = w1;
             }
           }
         }
