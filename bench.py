@@ -39,7 +39,7 @@ def read_peaks():
     return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
 
 
-KERNEL_SOURCES = {"prefill": "prefill_tc.cu", "compact": "compact.cu", "register": "register_mma.cu",
+KERNEL_SOURCES = {"prefill": "prefill_tc.cu", "compact": "compact.cu", "register": "register_mma.cu", "register_qkv": "register_qkv.cu",
                   "decode_compact": "decode_mma.cu", "decode_full": "decode_mma.cu"}
 
 
@@ -674,7 +674,8 @@ def main():
         for name, sec in tp.items():
             a = alg[name]
             parts[name] = {"ms_per_launch": sec * 1e3, "GB_s": a["bytes"] / sec / 1e9, "hbm_frac": a["bytes"] / sec / 1e9 / peaks["hbm_gbs"],
-                           "TFLOP_s": a["flops"] / sec / 1e12, "tensor_frac": a["flops"] / sec / 1e12 / peaks["tflops_burst"]}
+                           "TFLOP_s": a["flops"] / sec / 1e12, "tensor_frac": a["flops"] / sec / 1e12 / peaks["tflops_burst"],
+                           "traffic": traffic.get(name)}
 
     e2e = None
     if not args.no_e2e:
