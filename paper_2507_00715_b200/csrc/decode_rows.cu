@@ -20,8 +20,9 @@ namespace earn {
 namespace {
 using namespace dec;
 
-template <int D, int RT, int ST>   // RT warps = row tiles per CTA; ST ring stages, a multiple of RT
-__global__ void __launch_bounds__(RT * 32) decode_rows_kernel(DecodeArgs a) {
+// RT warps = row tiles per CTA; ST ring stages, a multiple of RT; MINB = CTAs per SM the register budget allows for
+template <int D, int RT, int ST, int MINB>
+__global__ void __launch_bounds__(RT * 32, MINB) decode_rows_kernel(DecodeArgs a) {
   using G = Geo<D>;
   constexpr int NT = RT * 32, CH = G::CH, SPW = ST / RT;   // SPW: ring stages a warp owns in phase 2
   static_assert(ST % RT == 0 && SPW >= 1 && NT % CH == 0, "ring slices");
@@ -72,6 +73,20 @@ __global__ void __launch_bounds__(RT * 32) decode_rows_kernel(DecodeArgs a) {
     cp_async_commit();
   }
 
+  // ---- where the generated tokens of this row tile's beams live: resolved now (lane -> positions lane, lane + 32,
+  // ... of the tile's list), so that the lineage look-ups are in flight together and under phase 1
+  const int w_lo = rm.row0 / g, w_hi = min((rm.row0 + 15) / g, W - 1);
+  const int n_priv = (active && split == 0) ? (w_hi - w_lo + 1) * step : 0, n_pt = (n_priv + KT - 1) / KT;
+  constexpr int NPRE = 4;   // rounds of 32 positions resolved ahead (8 tiles); later tiles are resolved as they come
+  int64_t pre[NPRE];        // element offset * 4 + tensor, -1: no such position
+#pragma unroll
+  for (int j = 0; j < NPRE; ++j) {
+    const int pk = j * 32 + lane;
+    int which = 1;
+    pre[j] = -1;
+    if (pk < n_priv) pre[j] = private_row<D>(a, b, kvh, w_lo, pk, which) * 4 + which;
+  }
+
   // ---- the Q fragments, while the first tiles are in flight
   RowTile<D> t;
   if (active) t.init(reinterpret_cast<const bf16*>(a.q), rm, lane);
@@ -99,17 +114,21 @@ __global__ void __launch_bounds__(RT * 32) decode_rows_kernel(DecodeArgs a) {
 
   // ---- phase 2 (split 0): the generated tokens of this row tile's beams, newest from k_new / v_new
   if (split == 0) {
-    const int w_lo = rm.row0 / g, w_hi = min((rm.row0 + 15) / g, W - 1);
-    const int n_priv = (w_hi - w_lo + 1) * step, n_pt = (n_priv + KT - 1) / KT;
     // positions of its list each of the lane's two rows may see: its own beam's `step` tokens
     const int vis0 = ((rm.row0 + (lane >> 2)) / g - w_lo) * step, vis1 = ((rm.row0 + (lane >> 2) + 8) / g - w_lo) * step;
     const uint32_t mine = ring + warp * SPW * G::STAGE_B;
     auto issue_private = [&](int tile, int stage) {
-      const int pk = tile * KT + lane;
-      int64_t off = -1;
-      int which = 1;
-      if (lane < KT && pk < n_priv) off = private_row<D>(a, b, kvh, w_lo, pk, which);
-      copy_resolved_tile<D>(mine + stage * G::STAGE_B, off, which, src, lane);
+      if (tile < 2 * NPRE) {   // tiles 2j and 2j + 1 were resolved by lanes 0..15 and 16..31 of round j
+        const int j = tile >> 1;
+        const int64_t e = j == 0 ? pre[0] : j == 1 ? pre[1] : j == 2 ? pre[2] : pre[3];
+        copy_resolved_tile<D>(mine + stage * G::STAGE_B, e < 0 ? -1 : e >> 2, (int)(e & 3), src, lane, (tile & 1) * 16);
+      } else {
+        const int pk = tile * KT + lane;
+        int64_t off = -1;
+        int which = 1;
+        if (lane < KT && pk < n_priv) off = private_row<D>(a, b, kvh, w_lo, pk, which);
+        copy_resolved_tile<D>(mine + stage * G::STAGE_B, off, which, src, lane);
+      }
     };
 #pragma unroll
     for (int s = 0; s < SPW - 1; ++s) {
@@ -144,14 +163,14 @@ __global__ void __launch_bounds__(RT * 32) decode_rows_kernel(DecodeArgs a) {
   }
 }
 
-template <int D, int RT, int ST>
+template <int D, int RT, int ST, int MINB>
 cudaError_t launch_rows(const DecodeArgs& a, cudaStream_t st) {
   constexpr int smem = ST * Geo<D>::STAGE_B;
-  cudaError_t e = ensure_dynamic_smem<decode_rows_kernel<D, RT, ST>>(smem);
+  cudaError_t e = ensure_dynamic_smem<decode_rows_kernel<D, RT, ST, MINB>>(smem);
   if (e != cudaSuccess) return e;
   const int splits = a.plan.n_splits > 0 ? a.plan.n_splits : 1;
   dim3 grid(a.Hkv, splits * ((a.plan.row_tiles + RT - 1) / RT), a.batch);
-  e = launch_pdl(decode_rows_kernel<D, RT, ST>, grid, dim3(RT * 32), smem, st, a);
+  e = launch_pdl(decode_rows_kernel<D, RT, ST, MINB>, grid, dim3(RT * 32), smem, st, a);
   note_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -159,9 +178,16 @@ cudaError_t launch_rows(const DecodeArgs& a, cudaStream_t st) {
 }  // namespace
 
 cudaError_t launch_decode_rows(const DecodeArgs& a, cudaStream_t st) {
-  const bool two = a.plan.row_tiles == 2;
-  if (a.D == 64) return two ? launch_rows<64, 2, 6>(a, st) : launch_rows<64, 4, 8>(a, st);
-  return two ? launch_rows<128, 2, 6>(a, st) : launch_rows<128, 4, 8>(a, st);
+  if (a.plan.row_tiles > 2) return a.D == 64 ? launch_rows<64, 4, 8, 1>(a, st) : launch_rows<128, 4, 8, 1>(a, st);
+  // Two row tiles (17 to 32 query rows per kv head, e.g. 20 beams of a multi-head model).  With a six-stage ring
+  // four CTAs fit an SM; a launch with more CTAs than that runs in waves, each paying the whole latency chain of a
+  // CTA, so it takes a four-stage ring and a register budget that fit six.  Measured on B200, 24 sequences x 32 kv
+  // heads x 20 beams (768 CTAs): 26.7 -> 17.5 us per compact-cache layer, 42.4 -> 30.8 us per prompt-cache layer;
+  // with few CTAs (8 long sequences, split) the deeper ring is the faster one, 49.8 against 54.0 us.
+  const long ctas = (long)a.Hkv * (a.plan.n_splits > 0 ? a.plan.n_splits : 1) * a.batch;
+  const bool many = ctas > 4L * 148;
+  if (a.D == 64) return many ? launch_rows<64, 2, 4, 6>(a, st) : launch_rows<64, 2, 6, 1>(a, st);
+  return many ? launch_rows<128, 2, 4, 6>(a, st) : launch_rows<128, 2, 6, 1>(a, st);
 }
 
 }  // namespace earn

@@ -277,18 +277,19 @@ struct Sources {
   const bf16* v[3];
 };
 
-// Copy one tile whose rows were resolved one per lane (lane i < KT holds the element offset `off` of position i's
-// row, -1 for "no such position", and the tensor `which`): the copying lanes fetch offset and tensor by shuffle.
-// stage = shared-memory address of the K tile; the V tile follows it.  Missing rows are zero-filled.
+// Copy one tile whose rows were resolved one per lane (lane lane_base + i, i < KT, holds the element offset `off` of
+// position i's row, -1 for "no such position", and the tensor `which`): the copying lanes fetch offset and tensor by
+// shuffle.  stage = shared-memory address of the K tile; the V tile follows it.  Missing rows are zero-filled.
 template <int D>
-__device__ __forceinline__ void copy_resolved_tile(uint32_t stage, int64_t off, int which, const Sources& src, int lane) {
+__device__ __forceinline__ void copy_resolved_tile(uint32_t stage, int64_t off, int which, const Sources& src, int lane,
+                                                   int lane_base = 0) {
   using G = Geo<D>;
   const int ch = lane % G::CH, r0 = lane / G::CH;
   const uint32_t kdst = stage + (uint32_t)r0 * G::PITCH + (uint32_t)ch * 16, vdst = kdst + G::TILE_B;
 #pragma unroll
   for (int i = 0; i < KT / G::RPI; ++i) {
-    const int64_t o_r = __shfl_sync(0xffffffffu, off, r0 + i * G::RPI);
-    const int w_r = __shfl_sync(0xffffffffu, which, r0 + i * G::RPI);
+    const int64_t o_r = __shfl_sync(0xffffffffu, off, lane_base + r0 + i * G::RPI);
+    const int w_r = __shfl_sync(0xffffffffu, which, lane_base + r0 + i * G::RPI);
     const bf16* ks = (w_r == 0 ? src.k[0] : w_r == 1 ? src.k[1] : src.k[2]) + (o_r < 0 ? 0 : o_r) + ch * 8;
     const bf16* vs = (w_r == 0 ? src.v[0] : w_r == 1 ? src.v[1] : src.v[2]) + (o_r < 0 ? 0 : o_r) + ch * 8;
     const int bytes = o_r < 0 ? 0 : 16;   // 0: nothing is read, the 16 destination bytes become zero
@@ -298,23 +299,46 @@ __device__ __forceinline__ void copy_resolved_tile(uint32_t stage, int64_t off, 
 }
 
 // Eq. 4, append: store the new K/V row of every beam whose first query row lies in rows row0 .. row0+15
-// (`n_threads` threads with index `tid` share the copy).
+// (`n_threads` threads with index `tid` share the copy).  The 16-byte pieces are fetched eight at a time before any
+// of them is stored: one round trip to memory per eight pieces instead of one per piece.
 template <int D>
 __device__ __forceinline__ void append_new_rows(const DecodeArgs& a, const RowMap& rm, int tid, int n_threads) {
-  constexpr int CH = Geo<D>::CH;
+  constexpr int CH = Geo<D>::CH, BATCH = 8;
   const bf16* kn = reinterpret_cast<const bf16*>(a.k_new);
   const bf16* vn = reinterpret_cast<const bf16*>(a.v_new);
   bf16* kp = reinterpret_cast<bf16*>(a.k_priv);
   bf16* vp = reinterpret_cast<bf16*>(a.v_priv);
-  const int w_lo = rm.row0 / rm.g, w_hi = min((rm.row0 + 15) / rm.g, rm.W - 1);
-  for (int w = w_lo; w <= w_hi; ++w) {
-    if (w * rm.g < rm.row0) continue;   // that beam's first row belongs to the previous row tile
-    const int64_t j = (int64_t)rm.b * rm.W + w;
-    const int64_t src = (j * a.Hkv + rm.kvh) * D, dst = ((j * a.max_new + (a.step - 1)) * a.Hkv + rm.kvh) * D;
-    for (int i = tid; i < 2 * CH; i += n_threads) {
-      const bf16* s = (i < CH ? kn : vn) + src + (i % CH) * 8;
-      bf16* d = (i < CH ? kp : vp) + dst + (i % CH) * 8;
-      *reinterpret_cast<uint4*>(d) = *reinterpret_cast<const uint4*>(s);
+  const int w_first = (rm.row0 + rm.g - 1) / rm.g;   // a beam whose first row belongs to the previous tile is appended there
+  const int w_last = min((rm.row0 + 15) / rm.g, rm.W - 1);
+  const int n_items = max(w_last - w_first + 1, 0) * 2 * CH;   // item = (beam, K or V, 16-byte piece)
+  if (n_items <= n_threads) {   // one beam per tile and the like: a single piece per thread
+    if (tid < n_items) {
+      const int64_t j = (int64_t)rm.b * rm.W + w_first + tid / (2 * CH);
+      const int c = tid % (2 * CH);
+      *reinterpret_cast<uint4*>((c < CH ? kp : vp) + ((j * a.max_new + (a.step - 1)) * a.Hkv + rm.kvh) * D + (c % CH) * 8) =
+          *reinterpret_cast<const uint4*>((c < CH ? kn : vn) + (j * a.Hkv + rm.kvh) * D + (c % CH) * 8);
+    }
+    return;
+  }
+  for (int i0 = tid; i0 < n_items; i0 += BATCH * n_threads) {
+    uint4 r[BATCH];
+#pragma unroll
+    for (int u = 0; u < BATCH; ++u) {
+      const int i = i0 + u * n_threads;
+      if (i < n_items) {
+        const int64_t j = (int64_t)rm.b * rm.W + w_first + i / (2 * CH);
+        const int c = i % (2 * CH);
+        r[u] = __ldg(reinterpret_cast<const uint4*>((c < CH ? kn : vn) + (j * a.Hkv + rm.kvh) * D + (c % CH) * 8));
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < BATCH; ++u) {
+      const int i = i0 + u * n_threads;
+      if (i < n_items) {
+        const int64_t j = (int64_t)rm.b * rm.W + w_first + i / (2 * CH);
+        const int c = i % (2 * CH);
+        *reinterpret_cast<uint4*>((c < CH ? kp : vp) + ((j * a.max_new + (a.step - 1)) * a.Hkv + rm.kvh) * D + (c % CH) * 8) = r[u];
+      }
     }
   }
 }
