@@ -44,13 +44,22 @@ KERNEL_SOURCES = {"prefill": "prefill_tc.cu", "compact": "compact.cu", "register
 
 
 def source_digest(fname: str) -> str:
-    """Digest of a kernel's source: the .cu file and every shared header of csrc/ (a kernel changes with either)."""
-    import glob
+    """Digest of a kernel's source: the .cu file and every header of csrc/ it includes, directly or through another
+    header (a kernel changes with any of them, and with no other file)."""
     import hashlib
+    import re
     csrc = os.path.join(ROOT, "paper_2507_00715_b200", "csrc")
+    seen, todo = [], [fname]
+    while todo:
+        name = todo.pop()
+        if name in seen or not os.path.exists(os.path.join(csrc, name)):
+            continue
+        seen.append(name)
+        with open(os.path.join(csrc, name)) as f:
+            todo += re.findall(r'^\s*#include\s+"([^"]+)"', f.read(), flags=re.M)
     h = hashlib.sha256()
-    for path in [os.path.join(csrc, fname)] + sorted(glob.glob(os.path.join(csrc, "*.cuh"))):
-        with open(path, "rb") as f:
+    for name in [fname] + sorted(n for n in seen if n != fname):
+        with open(os.path.join(csrc, name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()[:12]
 
