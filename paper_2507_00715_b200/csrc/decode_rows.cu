@@ -178,7 +178,8 @@ cudaError_t launch_rows(const DecodeArgs& a, cudaStream_t st) {
 }  // namespace
 
 cudaError_t launch_decode_rows(const DecodeArgs& a, cudaStream_t st) {
-  if (a.plan.row_tiles > 2) return a.D == 64 ? launch_rows<64, 4, 8, 1>(a, st) : launch_rows<128, 4, 8, 1>(a, st);
+  // four warps, eight stages: 68 KB of shared memory allow three CTAs per SM; hold the registers to that too
+  if (a.plan.row_tiles > 2) return a.D == 64 ? launch_rows<64, 4, 8, 3>(a, st) : launch_rows<128, 4, 8, 3>(a, st);
   // Two row tiles (17 to 32 query rows per kv head, e.g. 20 beams of a multi-head model).  With a six-stage ring
   // four CTAs fit an SM; a launch with more CTAs than that runs in waves, each paying the whole latency chain of a
   // CTA, so it takes a four-stage ring and a register budget that fit six.  Measured on B200, 24 sequences x 32 kv
@@ -186,8 +187,8 @@ cudaError_t launch_decode_rows(const DecodeArgs& a, cudaStream_t st) {
   // with few CTAs (8 long sequences, split) the deeper ring is the faster one, 49.8 against 54.0 us.
   const long ctas = (long)a.Hkv * (a.plan.n_splits > 0 ? a.plan.n_splits : 1) * a.batch;
   const bool many = ctas > 4L * 148;
-  if (a.D == 64) return many ? launch_rows<64, 2, 4, 6>(a, st) : launch_rows<64, 2, 6, 1>(a, st);
-  return many ? launch_rows<128, 2, 4, 6>(a, st) : launch_rows<128, 2, 6, 1>(a, st);
+  if (a.D == 64) return many ? launch_rows<64, 2, 4, 6>(a, st) : launch_rows<64, 2, 6, 4>(a, st);
+  return many ? launch_rows<128, 2, 4, 6>(a, st) : launch_rows<128, 2, 6, 4>(a, st);
 }
 
 }  // namespace earn
