@@ -298,6 +298,33 @@ __device__ __forceinline__ void copy_resolved_tile(uint32_t stage, int64_t off, 
   }
 }
 
+// Eq. 4, append, for the common case of at most one 16-byte piece per thread (one beam per row tile): fetch() early,
+// store() after the key loop, so that the round trip of the fetch hides under the loop.  When the row tile holds more
+// pieces than threads, active() is false and the caller falls back on append_new_rows().
+template <int D>
+struct AppendOne {
+  uint4 piece;
+  int64_t dst;      // element offset in the private segment, -1: nothing to store
+  bool is_v, single;
+  __device__ __forceinline__ void fetch(const DecodeArgs& a, const RowMap& rm, int tid, int n_threads, bool enabled) {
+    constexpr int CH = Geo<D>::CH;
+    const int w_first = (rm.row0 + rm.g - 1) / rm.g, w_last = min((rm.row0 + 15) / rm.g, rm.W - 1);
+    const int n_items = max(w_last - w_first + 1, 0) * 2 * CH;
+    single = n_items <= n_threads;
+    dst = -1;
+    if (enabled && single && tid < n_items) {
+      const int64_t j = (int64_t)rm.b * rm.W + w_first + tid / (2 * CH);
+      const int c = tid % (2 * CH);
+      is_v = c >= CH;
+      piece = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16*>(is_v ? a.v_new : a.k_new) + (j * a.Hkv + rm.kvh) * D + (c % CH) * 8);
+      dst = ((j * a.max_new + (a.step - 1)) * a.Hkv + rm.kvh) * D + (c % CH) * 8;
+    }
+  }
+  __device__ __forceinline__ void store(const DecodeArgs& a) const {
+    if (dst >= 0) *reinterpret_cast<uint4*>(reinterpret_cast<bf16*>(is_v ? a.v_priv : a.k_priv) + dst) = piece;
+  }
+};
+
 // Eq. 4, append: store the new K/V row of every beam whose first query row lies in rows row0 .. row0+15
 // (`n_threads` threads with index `tid` share the copy).  The 16-byte pieces are fetched eight at a time before any
 // of them is stored: one round trip to memory per eight pieces instead of one per piece.
