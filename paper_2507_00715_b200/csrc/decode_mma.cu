@@ -115,8 +115,15 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   };
 
   const int n_my = (n_tiles - warp + NWARPS - 1) / NWARPS;   // tiles warp, warp + NWARPS, ...
+  // Tiles in flight ahead of the one in use.  The streaming variants keep the ring full.  The five-stage variant
+  // (lists of three or four tiles, every CTA of the grid resident at once) starts with ONE tile: with 3.5 CTAs per
+  // SM asking for their whole list at the same moment the copies queue behind each other (a per-CTA timeline
+  // showed the fourth tile's cp.async issuing 3 us after the first), and the first tile's arithmetic might as well
+  // run under the rest of that queue: 7.55 -> 7.22 us per compact-cache layer at the 7B shapes (two and three
+  // tiles ahead measured 7.5).
+  constexpr int PRE = (NWARPS == 1 && STAGES == 5) ? 1 : STAGES - 1;
 #pragma unroll
-  for (int s = 0; s < STAGES - 1; ++s) {
+  for (int s = 0; s < PRE; ++s) {
     if (s < n_my) issue_tile(warp + s * NWARPS, s);
     cp_async_commit();
   }
@@ -137,10 +144,10 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   for (int it = 0; it < n_my; ++it) {
     const int stage = it % STAGES;
     {
-      const int nxt = it + STAGES - 1;   // refill the stage that was consumed in the previous iteration
+      const int nxt = it + PRE;          // into a stage that is free (consumed PRE + 1 <= STAGES iterations back, or never used)
       if (nxt < n_my) issue_tile(warp + nxt * NWARPS, nxt % STAGES);
       cp_async_commit();
-      cp_async_wait<STAGES - 1>();       // this lane's copies of tile `it` have landed ...
+      cp_async_wait<PRE>();              // this lane's copies of tile `it` have landed ...
       __syncwarp();                      // ... and so have every other lane's
     }
     const int tile = warp + it * NWARPS;
