@@ -24,14 +24,21 @@ namespace earn {
 namespace {
 using namespace ptx;
 
-constexpr int BM = 128, BN = 256, BK = 64, HD = 128;
-constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int NSTAGE = 4;
-constexpr int SMEM_BYTES = NSTAGE * STAGE_BYTES + 256 + 1024;
+constexpr int BM = 128, BK = 64, HD = 128;
+constexpr int A_BYTES = BM * BK * 2;
+// Tile geometry for an output tile of BN columns (256: two heads; 128: one head, for grids that would otherwise leave
+// most SMs without a tile): ring of 192 KB either way.
+template <int BN>
+struct Tile {
+  static constexpr int B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int NSTAGE = BN == 256 ? 4 : 6;
+  static constexpr int SMEM_BYTES = NSTAGE * STAGE_BYTES + 256 + 1024;
+  static constexpr int BAR_FULL = 0, BAR_EMPTY = NSTAGE, BAR_ACC_FULL = 2 * NSTAGE, BAR_ACC_EMPTY = BAR_ACC_FULL + 2,
+                       BAR_DRAIN = BAR_ACC_EMPTY + 2, N_BARS = BAR_DRAIN + 1;
+  static_assert(8 * N_BARS + 16 <= 256, "barrier block");
+};
 constexpr int THREADS = 256;
 constexpr long long WAIT_LIMIT = 2000000000LL;
-constexpr int BAR_FULL = 0, BAR_EMPTY = NSTAGE, BAR_ACC_FULL = 2 * NSTAGE, BAR_ACC_EMPTY = BAR_ACC_FULL + 2, BAR_DRAIN = BAR_ACC_EMPTY + 2,
-              N_BARS = BAR_DRAIN + 1;
 
 struct QkvParams {
   void* q_reg;
@@ -96,8 +103,13 @@ __global__ void __launch_bounds__(256) gather_norm_kernel(const __nv_bfloat16* x
 }
 
 // ---------------------------------------------------------------------------------------------------------------
+template <int BN>
 __global__ void __launch_bounds__(THREADS, 1)
 register_qkv_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, QkvParams p) {
+  using T = Tile<BN>;
+  constexpr int NSTAGE = T::NSTAGE, STAGE_BYTES = T::STAGE_BYTES, N_BARS = T::N_BARS;
+  constexpr int BAR_FULL = T::BAR_FULL, BAR_EMPTY = T::BAR_EMPTY, BAR_ACC_FULL = T::BAR_ACC_FULL,
+                BAR_ACC_EMPTY = T::BAR_ACC_EMPTY, BAR_DRAIN = T::BAR_DRAIN;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
@@ -122,7 +134,7 @@ register_qkv_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     tma_prefetch_desc(&map_b);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 2 * BN);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -281,7 +293,7 @@ register_qkv_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, (int32_t)EARN_ERR_TIMEOUT);
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem, 512);
+    tmem_dealloc(tmem, 2 * BN);
   }
 }
 
@@ -317,6 +329,19 @@ int sm_count_qkv() {
   return n;
 }
 
+template <int BN>
+cudaError_t launch_gemm(const RegisterQkvArgs& a, QkvParams p, int M, int N, int sms, cudaStream_t st) {
+  CUtensorMap ma, mb;
+  if (!make_map_2d(&ma, a.x_norm, M, a.d_model, BM) || !make_map_2d(&mb, a.w_qkv, N, a.d_model, BN)) return cudaErrorInvalidValue;
+  p.n_tiles = (N + BN - 1) / BN;
+  cudaError_t e = ensure_dynamic_smem<register_qkv_kernel<BN>>(Tile<BN>::SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  const int tiles = p.m_tiles * p.n_tiles;
+  e = launch_pdl(register_qkv_kernel<BN>, dim3(tiles < sms ? tiles : sms), dim3(THREADS), Tile<BN>::SMEM_BYTES, st, ma, mb, p);
+  note_launch();
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
 }  // namespace
 
 cudaError_t launch_register_qkv(const RegisterQkvArgs& a, cudaStream_t st) {
@@ -328,20 +353,16 @@ cudaError_t launch_register_qkv(const RegisterQkvArgs& a, cudaStream_t st) {
   note_launch();
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  CUtensorMap ma, mb;
-  if (!make_map_2d(&ma, a.x_norm, M, a.d_model, BM) || !make_map_2d(&mb, a.w_qkv, N, a.d_model, BN)) return cudaErrorInvalidValue;
   QkvParams p{};
   p.q_reg = a.q_reg; p.cache = a.cache; p.cu_seqlens = a.cu_seqlens; p.rope_cos = a.rope_cos; p.rope_sin = a.rope_sin;
   p.status = a.status; p.M = M; p.K = a.d_model; p.n_heads = n_heads; p.Hq = a.Hq; p.Hkv = a.Hkv; p.R = a.R;
   p.r_head = a.r_head; p.r_tail = a.r_tail; p.max_pos = a.max_pos;
   p.m_tiles = (M + BM - 1) / BM;
-  p.n_tiles = (N + BN - 1) / BN;
-  e = ensure_dynamic_smem<register_qkv_kernel>(SMEM_BYTES);
-  if (e != cudaSuccess) return e;
-  const int tiles = p.m_tiles * p.n_tiles, sms = sm_count_qkv();
-  e = launch_pdl(register_qkv_kernel, dim3(tiles < sms ? tiles : sms), dim3(THREADS), SMEM_BYTES, st, ma, mb, p);
-  note_launch();
-  return e != cudaSuccess ? e : cudaGetLastError();
+  // Two heads per tile unless that leaves most of the GPU idle: with few register rows (a batch of 24 prompts with
+  // two registers each is ONE row tile) the layer is a stream of W_qkv, and one-head tiles put twice as many SMs on it.
+  const int sms = sm_count_qkv();
+  const bool narrow = (long)p.m_tiles * ((N + 255) / 256) * 3 <= 2L * sms;
+  return narrow ? launch_gemm<128>(a, p, M, N, sms, st) : launch_gemm<256>(a, p, M, N, sms, st);
 }
 
 }  // namespace earn

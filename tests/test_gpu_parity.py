@@ -119,6 +119,15 @@ def test_beam_search_row_tiles_share_the_cache_pass():
                                           beams=7, decode_steps=3, r_head=4, r_tail=4))
 
 
+def test_two_row_tiles_on_a_grid_of_many_ctas_head_dim_64():
+    """20 beams of a multi-head model (two row tiles per kv head) over more (sequence, kv head) pairs than four CTAs
+    per SM hold: the launch takes the shallower ring with six CTAs per SM; head_dim 64; six decode steps, so the
+    private tiles outnumber a warp's ring slice; one register per side like the paper's own setting."""
+    lens = tuple(12 + (i * 7) % 30 for i in range(20))
+    run_workload_and_compare(BASE.replace(seed=27, head_dim=64, n_q_heads=32, n_kv_heads=32, lens=lens, batch=20, beams=20,
+                                          decode_steps=6, r_head=1, r_tail=1, n_layers=2, split_k=1), check_lse=False)
+
+
 def test_a_wait_that_runs_out_is_reported_and_the_context_survives():
     """Failure detection without a fault: a bounded device-side wait on a barrier nothing completes gives up after
     its limit, the kernel returns normally with EARN_ERR_TIMEOUT in the status word, and the library keeps working."""

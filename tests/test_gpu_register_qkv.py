@@ -83,7 +83,7 @@ def _run(w, compact=False, layers=None, sample=None, **session_kw):
 
 
 def test_small_ragged_one_tile():
-    """24 register rows (one ragged row tile), 8 heads, 8 k-blocks."""
+    """24 register rows (one ragged row tile), 8 heads, 8 k-blocks; few tiles, so one head per tile."""
     _run(_base())
 
 
@@ -103,6 +103,13 @@ def test_several_tiles_per_cta():
     w = _base(batch=40, lens=(), prompt_len=0, len_lo=40, len_hi=400, r_head=16, r_tail=16, n_q_heads=56, n_kv_heads=4,
               hidden=256, n_layers=2, seed=22)
     _run(w, sample=(0, 7, 39))
+
+
+def test_two_head_tiles_with_an_odd_head_count():
+    """1280 rows x 21 heads: enough tiles for the two-heads-per-tile kernel, whose last tile is half outside W_qkv."""
+    w = _base(batch=40, lens=(), prompt_len=0, len_lo=40, len_hi=400, r_head=16, r_tail=16, n_q_heads=15, n_kv_heads=3,
+              hidden=256, n_layers=2, seed=24)
+    _run(w, sample=(1, 20, 38))
 
 
 def test_deep_k():
