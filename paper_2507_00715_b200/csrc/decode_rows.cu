@@ -25,7 +25,7 @@ template <int D, int RT, int ST, int MINB>
 __global__ void __launch_bounds__(RT * 32, MINB) decode_rows_kernel(DecodeArgs a) {
   using G = Geo<D>;
   constexpr int NT = RT * 32, CH = G::CH, SPW = ST / RT;   // SPW: ring stages a warp owns in phase 2
-  static_assert(ST % RT == 0 && SPW >= 1 && NT % CH == 0, "ring slices");
+  static_assert(ST % RT == 0 && SPW >= 1 && NT % CH == 0 && ST >= 4, "ring slices");
   extern __shared__ __align__(128) uint8_t smem[];
   pdl_wait();   // everything below reads or writes global memory
 
@@ -68,7 +68,7 @@ __global__ void __launch_bounds__(RT * 32, MINB) decode_rows_kernel(DecodeArgs a
     }
   };
 #pragma unroll
-  for (int s = 0; s < ST - 1; ++s) {
+  for (int s = 0; s < ST - 2; ++s) {
     if (s < n_sh_tiles) issue_shared(s, s);
     cp_async_commit();
   }
@@ -91,17 +91,26 @@ __global__ void __launch_bounds__(RT * 32, MINB) decode_rows_kernel(DecodeArgs a
   RowTile<D> t;
   if (active) t.init(reinterpret_cast<const bf16*>(a.q), rm, lane);
 
-  for (int it = 0; it < n_sh_tiles; ++it) {
-    cp_async_wait<ST - 2>();   // this thread's copies of tile `it` have landed ...
-    __syncthreads();           // ... and everyone's; every warp is also done with tile it-1, whose stage is refilled next
-    {
-      const int nxt = it + ST - 1;
+  // two tiles per round: one block-wide barrier and one softmax step per 32 positions
+  for (int it = 0; it < n_sh_tiles; it += 2) {
+    cp_async_wait<ST - 4>();   // this thread's copies of tiles it and it+1 have landed ...
+    __syncthreads();           // ... and everyone's; every warp is also done with tiles it-2 and it-1, whose stages are refilled next
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int nxt = it + ST - 2 + u;
       if (nxt < n_sh_tiles) issue_shared(nxt, nxt % ST);
       cp_async_commit();
     }
     if (active) {
       const uint32_t ks = ring + (it % ST) * G::STAGE_B, vs = ks + G::TILE_B;
-      t.attend(ks, vs, scale_log2, lane, (it + 1) * KT > n_shared, [&](int c, bool) { return it * KT + c < n_shared; });
+      const uint32_t ks2 = ring + ((it + 1) % ST) * G::STAGE_B, vs2 = ks2 + G::TILE_B;
+      if ((it + 2) * KT <= n_shared) {
+        t.attend2(ks, vs, ks2, vs2, scale_log2, lane);
+      } else {
+        t.attend(ks, vs, scale_log2, lane, (it + 1) * KT > n_shared, [&](int c, bool) { return it * KT + c < n_shared; });
+        if (it + 1 < n_sh_tiles)
+          t.attend(ks2, vs2, scale_log2, lane, true, [&](int c, bool) { return (it + 1) * KT + c < n_shared; });
+      }
     }
   }
   cp_async_wait<0>();

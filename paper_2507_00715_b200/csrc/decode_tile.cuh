@@ -128,6 +128,68 @@ struct RowTile {
     }
   }
 
+  // Two whole tiles (2 * KT positions, every one visible to every row) in one softmax step: four independent chains
+  // of MMAs instead of two, one rescale of the accumulator and one round of quad shuffles per 32 positions.
+  __device__ __forceinline__ void attend2(uint32_t ksa, uint32_t vsa, uint32_t ksb, uint32_t vsb, float scale_log2, int lane) {
+    constexpr int PITCH = Geo<D>::PITCH;
+    const int mat = lane >> 3;
+    const uint32_t k_lane = (uint32_t)(((mat >> 1) << 3) + (lane & 7)) * PITCH + (uint32_t)(mat & 1) * 16;
+    const uint32_t v_lane = (uint32_t)(((mat & 1) << 3) + (lane & 7)) * PITCH + (uint32_t)(mat >> 1) * 16;
+    float s[4][4];
+#pragma unroll
+    for (int n = 0; n < 4; ++n) s[n][0] = s[n][1] = s[n][2] = s[n][3] = 0.f;
+#pragma unroll
+    for (int kk = 0; kk < KSTEPS; ++kk) {
+      uint32_t b0, b1, b2, b3, c0, c1, c2_, c3;
+      ldsm_x4(ksa + k_lane + kk * 32, b0, b1, b2, b3);
+      ldsm_x4(ksb + k_lane + kk * 32, c0, c1, c2_, c3);
+      mma_bf16(s[0], qf[kk], b0, b1);
+      mma_bf16(s[1], qf[kk], b2, b3);
+      mma_bf16(s[2], qf[kk], c0, c1);
+      mma_bf16(s[3], qf[kk], c2_, c3);
+    }
+    float mx0 = fmaxf(fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1])), fmaxf(fmaxf(s[2][0], s[2][1]), fmaxf(s[3][0], s[3][1])));
+    float mx1 = fmaxf(fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3])), fmaxf(fmaxf(s[2][2], s[2][3]), fmaxf(s[3][2], s[3][3])));
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+    const float mn0 = fmaxf(m0, mx0 * scale_log2), mn1 = fmaxf(m1, mx1 * scale_log2);   // finite: every position is visible
+    const float al0 = ex2(m0 - mn0), al1 = ex2(m1 - mn1);
+    const bool grew = (mn0 != m0) || (mn1 != m1);
+    m0 = mn0;
+    m1 = mn1;
+    uint32_t pf[2][4];
+    {
+      float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+      for (int n = 0; n < 4; ++n) {
+        const float p0 = ex2(fmaf(s[n][0], scale_log2, -mn0)), p1 = ex2(fmaf(s[n][1], scale_log2, -mn0));
+        const float p2 = ex2(fmaf(s[n][2], scale_log2, -mn1)), p3 = ex2(fmaf(s[n][3], scale_log2, -mn1));
+        sum0 += p0 + p1;
+        sum1 += p2 + p3;
+        pf[n >> 1][(n & 1) * 2] = pack2(p0, p1);
+        pf[n >> 1][(n & 1) * 2 + 1] = pack2(p2, p3);
+      }
+      l0 = l0 * al0 + sum0;
+      l1 = l1 * al1 + sum1;
+    }
+    if (__any_sync(0xffffffffu, grew)) {
+#pragma unroll
+      for (int n = 0; n < NTILES; ++n) { o[n][0] *= al0; o[n][1] *= al0; o[n][2] *= al1; o[n][3] *= al1; }
+    }
+#pragma unroll
+    for (int nn = 0; nn < NTILES / 2; ++nn) {
+      uint32_t b0, b1, b2, b3, c0, c1, c2_, c3;
+      ldsm_x4_t(vsa + v_lane + nn * 32, b0, b1, b2, b3);
+      ldsm_x4_t(vsb + v_lane + nn * 32, c0, c1, c2_, c3);
+      mma_bf16(o[2 * nn], pf[0], b0, b1);
+      mma_bf16(o[2 * nn + 1], pf[0], b2, b3);
+      mma_bf16(o[2 * nn], pf[1], c0, c1);
+      mma_bf16(o[2 * nn + 1], pf[1], c2_, c3);
+    }
+  }
+
   __device__ __forceinline__ void reduce_sums() {
     l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
     l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
