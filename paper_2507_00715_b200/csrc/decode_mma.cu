@@ -17,6 +17,10 @@
 // padded shared-memory tiles (a ring of four stages = 35 KB at head_dim 128, so six CTAs share an SM; two
 // stages for lists of at most two tiles).  Tile size, warps per CTA and ring depth were swept on B200 at
 // the 7B shapes: (16, 1, 4) gave 50.9 us per layer against 51.3-63.4 us for the other combinations.
+// A long list is then consumed two tiles at a time (one softmax step, one rescale of the accumulator and one
+// round of quad shuffles per 32 positions, four independent MMA chains instead of two): 49.6 -> 46.3 us per
+// prompt-cache layer at the 7B shapes, 6.0 TB/s.  Deeper rings behind the pairs were slower (five stages 48.0,
+// six 52.5, eight 76 us), three stages 56 us.
 // Rows that are an affine function of the list position (packed prompt K/V, identity page table)
 // take a fast path of pointer increments; any other tile (scattered pages, generated tokens
 // behind the lineage table, a ragged last tile) first resolves one row per lane and hands the row
@@ -38,6 +42,13 @@ using namespace dec;
 #define EARN_DECODE_STAGES 4
 #endif
 
+// how a CTA walks its key list
+enum Walk {
+  STREAM,   // one warp, a long list: tiles consumed two at a time behind a full ring
+  SHORT,    // one warp, a list of at most four tiles, every CTA of the grid resident at once: latency-bound
+  SHARED    // several warps deal the tiles round-robin and merge their states at the end
+};
+
 template <int D, int STAGES, int NWARPS>   // STAGES: cp.async ring depth per warp; NWARPS: warps per CTA, tiles dealt round-robin
 struct Smem {
   static constexpr int RING_B = NWARPS * STAGES * Geo<D>::STAGE_B;
@@ -45,8 +56,9 @@ struct Smem {
   static constexpr int BYTES = RING_B > MERGE_B ? RING_B : MERGE_B;
 };
 
-template <int D, int STAGES, int NWARPS>
+template <int D, int STAGES, int NWARPS, Walk WALK>
 __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
+  static_assert((WALK == SHARED) == (NWARPS > 1) && (WALK != STREAM || STAGES >= 3), "walk");
   using G = Geo<D>;
   constexpr int NTILES = D / 8, CH = G::CH, RPI = G::RPI, NIT = KT / RPI;
   extern __shared__ __align__(128) uint8_t smem[];
@@ -121,7 +133,10 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   // showed the fourth tile's cp.async issuing 3 us after the first), and the first tile's arithmetic might as well
   // run under the rest of that queue: 7.55 -> 7.22 us per compact-cache layer at the 7B shapes (two and three
   // tiles ahead measured 7.5).
-  constexpr int PRE = (NWARPS == 1 && STAGES == 5) ? 1 : STAGES - 1;
+  // The one-warp streaming variant consumes its tiles two at a time (one softmax step per 32 positions): the two
+  // tiles in use plus STAGES - 2 in flight.
+  constexpr bool PAIR = WALK == STREAM;
+  constexpr int PRE = (WALK == SHORT && STAGES == 5) ? 1 : PAIR ? STAGES - 2 : STAGES - 1;
 #pragma unroll
   for (int s = 0; s < PRE; ++s) {
     if (s < n_my) issue_tile(warp + s * NWARPS, s);
@@ -135,13 +150,40 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   // fetched here, behind the Q loads, and stored after the key loop: 7.9 -> 7.6 us per compact-cache layer at the 7B
   // shapes.  The streaming variant keeps fetch and store together after its loop (the extra live registers cost
   // it 1 to 3 %).
-  constexpr bool EARLY_APPEND = NWARPS == 1 && STAGES != EARN_DECODE_STAGES;
+  constexpr bool EARLY_APPEND = WALK == SHORT;
   AppendOne<D> app;
   if (EARLY_APPEND) app.fetch(a, rm, threadIdx.x, NWARPS * 32, split == 0);
   // list positions of the generated tokens each of the lane's two rows may see: its own beam's `step` tokens
   const int vis0 = n_shared + ((row0 + (lane >> 2)) / g - w_lo) * step, vis1 = n_shared + ((row0 + (lane >> 2) + 8) / g - w_lo) * step;
 
-  for (int it = 0; it < n_my; ++it) {
+  auto visible_in = [&](int tile) {
+    return [=](int c, bool second) {
+      const int p = tile * KT + c, v0 = second ? vis1 : vis0;
+      return p < n_shared || (p >= v0 && p < v0 + step && p < n_total);
+    };
+  };
+  if (PAIR) {
+    for (int it = 0; it < n_my; it += 2) {
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {   // into the two stages the previous round consumed (or that were never used)
+        const int nxt = it + PRE + u;
+        if (nxt < n_my) issue_tile(nxt, nxt % STAGES);
+        cp_async_commit();
+      }
+      cp_async_wait<PRE>();           // this lane's copies of tiles it and it+1 have landed ...
+      __syncwarp();                   // ... and so have every other lane's
+      const uint32_t ks = ring + (it % STAGES) * G::STAGE_B, vs = ks + G::TILE_B;
+      const uint32_t ks2 = ring + ((it + 1) % STAGES) * G::STAGE_B, vs2 = ks2 + G::TILE_B;
+      if ((it + 2) * KT <= n_shared) {
+        t.attend2(ks, vs, ks2, vs2, scale_log2, lane);
+      } else {
+        t.attend(ks, vs, scale_log2, lane, (it + 1) * KT > n_shared, visible_in(it));
+        if (it + 1 < n_my) t.attend(ks2, vs2, scale_log2, lane, true, visible_in(it + 1));
+      }
+      __syncwarp();   // every lane is done with these stages before the next round refills them
+    }
+  }
+  for (int it = 0; !PAIR && it < n_my; ++it) {
     const int stage = it % STAGES;
     {
       const int nxt = it + PRE;          // into a stage that is free (consumed PRE + 1 <= STAGES iterations back, or never used)
@@ -234,14 +276,14 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   }
 }
 
-template <int D, int ST, int NWARPS>
+template <int D, int ST, int NWARPS, Walk WALK>
 cudaError_t launch_d(const DecodeArgs& a, cudaStream_t st) {
   constexpr int smem = Smem<D, ST, NWARPS>::BYTES;
-  cudaError_t e = ensure_dynamic_smem<decode_mma_kernel<D, ST, NWARPS>>(smem);
+  cudaError_t e = ensure_dynamic_smem<decode_mma_kernel<D, ST, NWARPS, WALK>>(smem);
   if (e != cudaSuccess) return e;
   const int splits = a.plan.n_splits > 0 ? a.plan.n_splits : 1;
   dim3 grid(a.Hkv, splits * a.plan.row_tiles, a.batch);
-  e = launch_pdl(decode_mma_kernel<D, ST, NWARPS>, grid, dim3(NWARPS * 32), smem, st, a);
+  e = launch_pdl(decode_mma_kernel<D, ST, NWARPS, WALK>, grid, dim3(NWARPS * 32), smem, st, a);
   note_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -265,14 +307,14 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, int max_shared_len, cudaStrea
   // the tile that had to wait for a free stage cost about 1.5 us at the 7B shapes
   const bool two_tiles = unsplit && max_tiles <= 2, four_tiles = unsplit && max_tiles <= 4;
   if (a.D == 64)
-    return four_warps  ? launch_d<64, 2, 4>(a, st)
-           : two_tiles ? launch_d<64, 3, 1>(a, st)
-           : four_tiles ? launch_d<64, 5, 1>(a, st)
-                        : launch_d<64, EARN_DECODE_STAGES, 1>(a, st);
-  return four_warps  ? launch_d<128, 2, 4>(a, st)
-         : two_tiles ? launch_d<128, 3, 1>(a, st)
-         : four_tiles ? launch_d<128, 5, 1>(a, st)
-                      : launch_d<128, EARN_DECODE_STAGES, 1>(a, st);
+    return four_warps  ? launch_d<64, 2, 4, SHARED>(a, st)
+           : two_tiles ? launch_d<64, 3, 1, SHORT>(a, st)
+           : four_tiles ? launch_d<64, 5, 1, SHORT>(a, st)
+                        : launch_d<64, EARN_DECODE_STAGES, 1, STREAM>(a, st);
+  return four_warps  ? launch_d<128, 2, 4, SHARED>(a, st)
+         : two_tiles ? launch_d<128, 3, 1, SHORT>(a, st)
+         : four_tiles ? launch_d<128, 5, 1, SHORT>(a, st)
+                      : launch_d<128, EARN_DECODE_STAGES, 1, STREAM>(a, st);
 }
 
 }  // namespace earn
