@@ -45,7 +45,7 @@ using namespace dec;
 // how a CTA walks its key list
 enum Walk {
   STREAM,   // one warp, a long list: tiles consumed two at a time behind a full ring
-  SHORT,    // one warp, a list of at most four tiles, every CTA of the grid resident at once: latency-bound
+  SHORT,    // one warp, a list of at most two tiles: the whole list in flight from the start
   SHARED    // several warps deal the tiles round-robin and merge their states at the end
 };
 
@@ -127,16 +127,10 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   };
 
   const int n_my = (n_tiles - warp + NWARPS - 1) / NWARPS;   // tiles warp, warp + NWARPS, ...
-  // Tiles in flight ahead of the one in use.  The streaming variants keep the ring full.  The five-stage variant
-  // (lists of three or four tiles, every CTA of the grid resident at once) starts with ONE tile: with 3.5 CTAs per
-  // SM asking for their whole list at the same moment the copies queue behind each other (a per-CTA timeline
-  // showed the fourth tile's cp.async issuing 3 us after the first), and the first tile's arithmetic might as well
-  // run under the rest of that queue: 7.55 -> 7.22 us per compact-cache layer at the 7B shapes (two and three
-  // tiles ahead measured 7.5).
   // The one-warp streaming variant consumes its tiles two at a time (one softmax step per 32 positions): the two
   // tiles in use plus STAGES - 2 in flight.
   constexpr bool PAIR = WALK == STREAM;
-  constexpr int PRE = (WALK == SHORT && STAGES == 5) ? 1 : PAIR ? STAGES - 2 : STAGES - 1;
+  constexpr int PRE = PAIR ? STAGES - 2 : STAGES - 1;   // tiles in flight ahead of the one(s) in use
 #pragma unroll
   for (int s = 0; s < PRE; ++s) {
     if (s < n_my) issue_tile(warp + s * NWARPS, s);
@@ -146,13 +140,11 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   // ---- Q fragments, loaded while the first tiles are in flight
   RowTile<D> t;
   t.init(reinterpret_cast<const bf16*>(a.q), rm, lane);
-  // Eq. 4 append.  In the short-list variants (whole list in flight from the start; latency-bound) the new row is
-  // fetched here, behind the Q loads, and stored after the key loop: 7.9 -> 7.6 us per compact-cache layer at the 7B
-  // shapes.  The streaming variant keeps fetch and store together after its loop (the extra live registers cost
-  // it 1 to 3 %).
-  constexpr bool EARLY_APPEND = WALK == SHORT;
+  // Eq. 4 append: the new row is fetched here, behind the Q loads, and stored after the key loop, so that the round
+  // trip of the fetch hides under the loop (7.9 -> 7.6 us per compact-cache layer at the 7B shapes, 11.9 -> 11.5 us
+  // per prompt-cache layer at the 1.5B shapes).
   AppendOne<D> app;
-  if (EARLY_APPEND) app.fetch(a, rm, threadIdx.x, NWARPS * 32, split == 0);
+  app.fetch(a, rm, threadIdx.x, NWARPS * 32, split == 0);
   // list positions of the generated tokens each of the lane's two rows may see: its own beam's `step` tokens
   const int vis0 = n_shared + ((row0 + (lane >> 2)) / g - w_lo) * step, vis1 = n_shared + ((row0 + (lane >> 2) + 8) / g - w_lo) * step;
 
@@ -205,7 +197,7 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   // ---- Eq. 4: append.  Split 0 stores the new K/V row of every beam whose first query row is in this tile.  Nothing
   // in this launch reads those rows (the newest token came straight from k_new / v_new), so the store waits until
   // here: a whole load-then-store round trip ahead of the Q loads delayed them by more than a microsecond.
-  if (EARLY_APPEND && app.single) app.store(a);
+  if (app.single) app.store(a);
   else if (split == 0) append_new_rows<D>(a, rm, threadIdx.x, NWARPS * 32);
   // The next kernel on the stream may be scheduled from here on (once every CTA of this grid is past its key
   // loop): releasing it earlier let its CTAs pile up on whichever SMs had room and unbalanced the next launch
@@ -303,17 +295,14 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, int max_shared_len, cudaStrea
   const long ctas = (long)(a.plan.n_splits > 0 ? a.plan.n_splits : 1) * a.plan.row_tiles * a.Hkv * a.batch;
   const bool unsplit = a.plan.n_splits <= 1;
   const bool four_warps = unsplit && max_tiles <= 16 && ctas < 148;
-  // a ring of n+1 stages has a whole list of n tiles in flight from the start: short lists are latency-bound and
-  // the tile that had to wait for a free stage cost about 1.5 us at the 7B shapes
-  const bool two_tiles = unsplit && max_tiles <= 2, four_tiles = unsplit && max_tiles <= 4;
+  // a list of one or two tiles goes into a three-stage ring whole; anything longer is walked in pairs
+  const bool two_tiles = unsplit && max_tiles <= 2;
   if (a.D == 64)
     return four_warps  ? launch_d<64, 2, 4, SHARED>(a, st)
            : two_tiles ? launch_d<64, 3, 1, SHORT>(a, st)
-           : four_tiles ? launch_d<64, 5, 1, SHORT>(a, st)
                         : launch_d<64, EARN_DECODE_STAGES, 1, STREAM>(a, st);
   return four_warps  ? launch_d<128, 2, 4, SHARED>(a, st)
          : two_tiles ? launch_d<128, 3, 1, SHORT>(a, st)
-         : four_tiles ? launch_d<128, 5, 1, SHORT>(a, st)
                       : launch_d<128, EARN_DECODE_STAGES, 1, STREAM>(a, st);
 }
 
