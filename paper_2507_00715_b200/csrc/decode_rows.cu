@@ -58,8 +58,9 @@ __global__ void __launch_bounds__(RT * 32, MINB) decode_rows_kernel(DecodeArgs a
   auto issue_shared = [&](int tile, int stage) {
     const uint32_t kdst = ring + stage * G::STAGE_B + (uint32_t)c_t * 16, vdst = kdst + G::TILE_B;
 #pragma unroll
-    for (int i = 0; i < KT * CH / NT; ++i) {
+    for (int i = 0; i < (KT + NT / CH - 1) / (NT / CH); ++i) {   // NT / CH rows per pass; the last pass may be partial
       const int r = r_t + i * (NT / CH), p = tile * KT + r;
+      if (KT % (NT / CH) != 0 && r >= KT) break;
       const bool ok = p < n_shared;
       const int64_t row = !ok ? 0 : affine ? row_base + key_begin + p : key_row(a.src, b, key_begin + p);
       const int64_t off = (row * a.Hkv + kvh) * D + c_t * 8;
@@ -188,7 +189,19 @@ cudaError_t launch_rows(const DecodeArgs& a, cudaStream_t st) {
 
 cudaError_t launch_decode_rows(const DecodeArgs& a, cudaStream_t st) {
   // four warps, eight stages: 68 KB of shared memory allow three CTAs per SM; hold the registers to that too
-  if (a.plan.row_tiles > 2) return a.D == 64 ? launch_rows<64, 4, 8, 3>(a, st) : launch_rows<128, 4, 8, 3>(a, st);
+  if (a.plan.row_tiles > 2) {
+    // Three row tiles per CTA (96 threads, six stages, four CTAs per SM) when that leaves fewer warps without a row
+    // tile than four would (3, 5, 6 and 9 row tiles) and the shared segment is short, so that the launch is bound by
+    // the latency chain of a CTA and by how many CTAs are resident, not by streaming.  Measured on B200: 48
+    // sequences x 4 kv heads x 140 rows (20 beams, group of 7), 50-200 token prompts: 16.3 -> 10.3 us per
+    // compact-cache layer, 27.0 -> 20.2 us per prompt-cache layer; 128 sequences x 8 kv heads x 40 rows: 42.7 -> 34.7
+    // us per compact-cache layer, but 201 -> 208 us per prompt-cache layer of up to 2048 tokens, which therefore
+    // keeps four warps and the eight-stage ring.
+    const int rt = a.plan.row_tiles, idle3 = (rt + 2) / 3 * 3 - rt, idle4 = (rt + 3) / 4 * 4 - rt;
+    const bool three = idle3 < idle4 && a.plan.chunk <= 512;
+    if (three) return a.D == 64 ? launch_rows<64, 3, 6, 4>(a, st) : launch_rows<128, 3, 6, 4>(a, st);
+    return a.D == 64 ? launch_rows<64, 4, 8, 3>(a, st) : launch_rows<128, 4, 8, 3>(a, st);
+  }
   // Two row tiles (17 to 32 query rows per kv head, e.g. 20 beams of a multi-head model).  With a six-stage ring
   // four CTAs fit an SM; a launch with more CTAs than that runs in waves, each paying the whole latency chain of a
   // CTA, so it takes a four-stage ring and a register budget that fit six.  Measured on B200, 24 sequences x 32 kv
