@@ -67,7 +67,7 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // kv heads vary fastest over the grid: the CTAs that read the same rows of the packed K/V tensors (one 256-byte
   // slice each of a 2 KB row) start next to each other and walk those rows together
-  const int b = blockIdx.z, kvh = blockIdx.x;
+  const int b = a.by_length ? sequence_of_rank(a.cu_seqlens, a.batch, blockIdx.z, lane) : (int)blockIdx.z, kvh = blockIdx.x;
   const int row_tiles = a.plan.row_tiles;
   const int split = blockIdx.y / row_tiles, row_tile = blockIdx.y % row_tiles;
   RowMap rm;

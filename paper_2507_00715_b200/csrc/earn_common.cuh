@@ -136,6 +136,7 @@ struct DecodeArgs {
   DecodePlan plan;
   int batch, beams, max_new, step, Hq, Hkv, D, dtype;
   float scale;
+  int by_length;               // bf16 kernels: grid index z is a RANK in the order of decreasing shared length, not a sequence
 };
 cudaError_t launch_decode_simt(const DecodeArgs& a, cudaStream_t st);   // fp32 debug path
 // bf16: cp.async ring + mma.sync; max_shared_len = longest shared segment of the batch (picks the ring depth)

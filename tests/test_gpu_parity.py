@@ -128,6 +128,15 @@ def test_two_row_tiles_on_a_grid_of_many_ctas_head_dim_64():
                                           decode_steps=6, r_head=1, r_tail=1, n_layers=2, split_k=1), check_lse=False)
 
 
+def test_long_uneven_prompts_are_decoded_longest_first():
+    """Prompt-cache decode of a batch whose prompts are long and uneven hands its CTAs out by decreasing length (the
+    grid index is a rank, the kernel looks the sequence up): equal lengths in the batch exercise the tie rule; one
+    beam (one row tile) and five beams (several row tiles)."""
+    w = BASE.replace(seed=28, lens=(1200, 90, 400, 1200, 33, 1024), batch=6, n_layers=2, split_k=1, decode_steps=2)
+    run_workload_and_compare(w, check_lse=False)
+    run_workload_and_compare(w.replace(seed=29, beams=5), check_lse=False)
+
+
 def test_a_wait_that_runs_out_is_reported_and_the_context_survives():
     """Failure detection without a fault: a bounded device-side wait on a barrier nothing completes gives up after
     its limit, the kernel returns normally with EARN_ERR_TIMEOUT in the status word, and the library keeps working."""
