@@ -67,7 +67,9 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // kv heads vary fastest over the grid: the CTAs that read the same rows of the packed K/V tensors (one 256-byte
   // slice each of a 2 KB row) start next to each other and walk those rows together
-  const int b = a.by_length ? sequence_of_rank(a.cu_seqlens, a.batch, blockIdx.z, lane) : (int)blockIdx.z, kvh = blockIdx.x;
+  // CTAs are handed out in grid order: with an order table the longest sequences start first and the launch does
+  // not end on a long sequence that started late
+  const int b = a.order ? a.order[blockIdx.z] : (int)blockIdx.z, kvh = blockIdx.x;
   const int row_tiles = a.plan.row_tiles;
   const int split = blockIdx.y / row_tiles, row_tile = blockIdx.y % row_tiles;
   RowMap rm;
@@ -280,7 +282,27 @@ cudaError_t launch_d(const DecodeArgs& a, cudaStream_t st) {
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
+// order[rank] = sequence, longest prompt first (ties by index): thread c counts the sequences ahead of sequence c
+__global__ void __launch_bounds__(1024) decode_order_kernel(const int32_t* cu_seqlens, int batch, int32_t* order) {
+  __shared__ int len[1024];
+  pdl_wait();   // the table may still be read by the kernel before this one
+  const int c = threadIdx.x;
+  if (c < batch) len[c] = cu_seqlens[c + 1] - cu_seqlens[c];
+  __syncthreads();
+  pdl_launch_dependents();
+  if (c >= batch) return;
+  int ahead = 0;
+  for (int j = 0; j < batch; ++j) ahead += (len[j] > len[c]) || (len[j] == len[c] && j < c);
+  order[ahead] = c;
+}
+
 }  // namespace
+
+cudaError_t launch_decode_order(const int32_t* cu_seqlens, int batch, int32_t* order, cudaStream_t st) {
+  const cudaError_t e = launch_pdl(decode_order_kernel, dim3(1), dim3((batch + 31) / 32 * 32), 0, st, cu_seqlens, batch, order);
+  note_launch();
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
 
 cudaError_t launch_decode_mma(const DecodeArgs& a, int max_shared_len, cudaStream_t st) {
   // Several row tiles (beams x group size > 16): the row tiles of a CTA share one pass over the shared segment.

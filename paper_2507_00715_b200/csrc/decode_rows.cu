@@ -30,7 +30,9 @@ __global__ void __launch_bounds__(RT * 32, MINB) decode_rows_kernel(DecodeArgs a
   pdl_wait();   // everything below reads or writes global memory
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b = a.by_length ? sequence_of_rank(a.cu_seqlens, a.batch, blockIdx.z, lane) : (int)blockIdx.z, kvh = blockIdx.x;
+  // CTAs are handed out in grid order: with an order table the longest sequences start first and the launch does
+  // not end on a long sequence that started late
+  const int b = a.order ? a.order[blockIdx.z] : (int)blockIdx.z, kvh = blockIdx.x;
   const int row_groups = (a.plan.row_tiles + RT - 1) / RT;
   const int split = blockIdx.y / row_groups, row_tile = (blockIdx.y % row_groups) * RT + warp;
   const bool active = row_tile < a.plan.row_tiles;   // a warp without a row tile still helps with the copies

@@ -22,27 +22,6 @@ struct Geo {
   static constexpr int RPI = 32 / CH;           // rows one 16-byte access of a whole warp covers
 };
 
-// The sequence whose prompt is the rank-th longest of the batch (ties by index), found by one warp from cu_seqlens
-// alone: lane l ranks candidates l, l + 32, ... against every length and the search stops at the first hit.  CTAs are
-// handed out in grid order, so a grid whose z index is such a rank starts its longest sequences first and the launch
-// does not end on a long sequence that started late.  O(batch^2 / 32) per warp: for batches of a few hundred
-// sequences only.  (Keeping every candidate's key in registers and broadcasting the keys by shuffle does a quarter of
-// the comparisons but measured slower inside these register-bound kernels: 192-196 against 186 us per layer.)
-__device__ __forceinline__ int sequence_of_rank(const int32_t* cu_seqlens, int batch, int rank, int lane) {
-  for (int c0 = 0; c0 < batch; c0 += 32) {
-    const int cand = c0 + lane;
-    const int len_c = cand < batch ? cu_seqlens[cand + 1] - cu_seqlens[cand] : -1;
-    int ahead = 0;   // sequences that come before the candidate in the order
-    for (int j = 0; j < batch; ++j) {
-      const int len_j = cu_seqlens[j + 1] - cu_seqlens[j];
-      ahead += (len_j > len_c) || (len_j == len_c && j < cand);
-    }
-    const unsigned hit = __ballot_sync(0xffffffffu, cand < batch && ahead == rank);
-    if (hit) return c0 + __ffs(hit) - 1;
-  }
-  return rank;   // not reached: ranks are a permutation of the sequences
-}
-
 // Which query rows a warp owns: rows row0 .. row0+15 of the W*g rows of one (sequence, kv head);
 // row rr is beam rr / g, head kvh*g + rr % g.
 struct RowMap {

@@ -321,16 +321,22 @@ earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* ba
   a.batch = batch->batch; a.beams = cache->beams; a.max_new = cache->max_new; a.step = step;
   a.Hq = model->n_q_heads; a.Hkv = model->n_kv_heads; a.D = model->head_dim; a.dtype = model->dtype;
   a.scale = scale_of(model);
-  // Prompt-cache layers of a ragged batch: hand the CTAs out longest sequence first.  Worth its look-up (a pass of
-  // every warp over cu_seqlens) when the prompts are long and uneven and the batch is a few hundred sequences at most.
-  a.by_length = 0;
-  if (early && batch->batch >= 2 && batch->batch <= 256 && batch->max_seqlen >= 1024) {
+  // Prompt-cache layers of a ragged batch: hand the CTAs out longest sequence first.  The order table (one small
+  // launch ahead of the decode kernel) lives in the workspace's prefill-plan area, which holds at least 16 bytes per
+  // sequence and is rewritten by every prefill call before it is read.  Worth it when the prompts are long and uneven.
+  a.order = nullptr;
+  if (early && model->dtype == EARN_BF16 && batch->batch >= 2 && batch->batch <= 1024 && batch->max_seqlen >= 1024 &&
+      prefill_plan_bytes(*batch) >= sizeof(int32_t) * (size_t)batch->batch) {   // (empty sequences have no plan entry)
     int mn = batch->max_seqlen;
     for (int i = 0; i < batch->batch; ++i) {
       const int len = batch->cu_seqlens_host[i + 1] - batch->cu_seqlens_host[i];
       mn = len < mn ? len : mn;
     }
-    a.by_length = (int64_t)batch->max_seqlen * 4 > (int64_t)mn * 5;   // longest more than 1.25 x shortest
+    if ((int64_t)batch->max_seqlen * 4 > (int64_t)mn * 5) {   // longest more than 1.25 x shortest
+      int32_t* order = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(workspace) + kStatusBytes);
+      if (launch_decode_order(batch->cu_seqlens, batch->batch, order, (cudaStream_t)stream) != cudaSuccess) return EARN_ERR_CUDA;
+      a.order = order;
+    }
   }
   const cudaError_t e = model->dtype == EARN_BF16 ? launch_decode_mma(a, early ? batch->max_seqlen : batch->n_head_reg + batch->n_tail_reg, (cudaStream_t)stream)
                                                    : launch_decode_simt(a, (cudaStream_t)stream);

@@ -136,13 +136,15 @@ struct DecodeArgs {
   DecodePlan plan;
   int batch, beams, max_new, step, Hq, Hkv, D, dtype;
   float scale;
-  int by_length;               // bf16 kernels: grid index z is a RANK in the order of decreasing shared length, not a sequence
+  const int32_t* order;        // bf16 kernels: if not null, grid index z is a rank and order[z] the sequence (longest shared segment first)
 };
 cudaError_t launch_decode_simt(const DecodeArgs& a, cudaStream_t st);   // fp32 debug path
 // bf16: cp.async ring + mma.sync; max_shared_len = longest shared segment of the batch (picks the ring depth)
 cudaError_t launch_decode_mma(const DecodeArgs& a, int max_shared_len, cudaStream_t st);
 // bf16, several row tiles (beams x group size > 16): the row tiles of a CTA share one pass over the shared segment
 cudaError_t launch_decode_rows(const DecodeArgs& a, cudaStream_t st);
+// order[rank] = sequence, by decreasing prompt length (ties by index); batch <= 1024
+cudaError_t launch_decode_order(const int32_t* cu_seqlens, int batch, int32_t* order, cudaStream_t st);
 
 struct CompactArgs {
   const void *k, *v, *q;
