@@ -130,8 +130,8 @@ def test_two_row_tiles_on_a_grid_of_many_ctas_head_dim_64():
 
 def test_long_uneven_prompts_are_decoded_longest_first():
     """Prompt-cache decode of a batch whose prompts are long and uneven hands its CTAs out by decreasing length (the
-    grid index is a rank, the kernel looks the sequence up): equal lengths in the batch exercise the tie rule; one
-    beam (one row tile) and five beams (several row tiles)."""
+    grid index is a rank; a small launch ahead of the kernel writes the rank -> sequence table): equal lengths in the
+    batch exercise the tie rule; one beam (one row tile) and five beams (several row tiles)."""
     w = BASE.replace(seed=28, lens=(1200, 90, 400, 1200, 33, 1024), batch=6, n_layers=2, split_k=1, decode_steps=2)
     run_workload_and_compare(w, check_lse=False)
     run_workload_and_compare(w.replace(seed=29, beams=5), check_lse=False)
