@@ -172,6 +172,9 @@ earn_status_t earn_register_attn(const earn_model_t* model, const earn_batch_t* 
  *   layer >= k : the R compact register rows of sequence b, then the step generated tokens of its lineage;
  *   layer <  k : all L_b prompt rows of sequence b read in place from k_full/v_full (device, packed like
  *                earn_prefill_attn's k and v; required), then the generated tokens.
+ * For a layer < k of a batch with long, uneven prompts (longest >= 1024 tokens and more than 1.25 times the shortest,
+ * at most 1024 sequences) one small extra kernel runs first: it writes, into the plan area of the workspace, the order
+ * in which the main kernel takes the sequences (longest first).
  * Errors: step outside [1, max_new], missing k_full for a layer < k -> INVALID_ARG. */
 earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, int32_t step,
                                const void* q, const void* k_new, const void* v_new,
