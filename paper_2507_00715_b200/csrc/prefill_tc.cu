@@ -44,17 +44,18 @@ constexpr long long WAIT_LIMIT = 2000000000LL;     // about one second of SM clo
 constexpr int NT = 2;   // M-tiles per work item
 
 struct Cfg {
-  static constexpr int NSTAGE = 5;                          // ring entries (K and V tiles alternate)
+  static constexpr int NSTAGE = 4;                          // ring entries (K and V tiles alternate); five measured the same
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_RING = OFF_Q + NT * TILE;
-  static constexpr int OFF_BAR = OFF_RING + NSTAGE * TILE;
+  static constexpr int OFF_OUT = OFF_RING + NSTAGE * TILE;  // per M-tile: one 128 x 64 bf16 block of O on its way out
+  static constexpr int OFF_BAR = OFF_OUT + NT * HALF;
   static constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;   // + alignment slack
   static constexpr int TMEM_COLS = NT * 256;                // S_x (and P_x over it) at x*128, O_x at (NT + x)*128
   static constexpr int THREADS = 32 * (4 + 4 * NT);
   // barriers
   static constexpr int BAR_FULL = 0, BAR_EMPTY = BAR_FULL + NSTAGE, BAR_QFULL = BAR_EMPTY + NSTAGE,
                        BAR_QFREE = BAR_QFULL + NT, BAR_S = BAR_QFREE + NT, BAR_P = BAR_S + NT, BAR_O = BAR_P + NT,
-                       BAR_DRAIN = BAR_O + NT, N_BARS = BAR_DRAIN + 1;
+                       BAR_OUT = BAR_O + NT, BAR_DRAIN = BAR_OUT + NT, N_BARS = BAR_DRAIN + 1;
   static_assert(8 * N_BARS + 16 <= 512, "barrier block");
 };
 
@@ -120,7 +121,7 @@ __device__ __forceinline__ void add2(float& d0, float& d1, float a0, float a1) {
 template <bool PAIR_TILES>
 __global__ void __launch_bounds__(Cfg::THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                  const __grid_constant__ CUtensorMap map_v, TcParams p) {
+                  const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_o, TcParams p) {
   using C = Cfg;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;    // swizzled tiles need 1024-byte alignment
@@ -143,6 +144,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       mbar_init(bar(C::BAR_S + x), 1);
       mbar_init(bar(C::BAR_P + x), 128);
       mbar_init(bar(C::BAR_O + x), 1);
+      mbar_init(bar(C::BAR_OUT + x), 128);
     }
     mbar_init(bar(C::BAR_DRAIN), 1);
     *abort_flag = 0;
@@ -150,6 +152,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     tma_prefetch_desc(&map_q);
     tma_prefetch_desc(&map_k);
     tma_prefetch_desc(&map_v);
+    tma_prefetch_desc(&map_o);
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), C::TMEM_COLS);
@@ -315,8 +318,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const uint32_t t_s = tmem + ((uint32_t)(wq * 32) << 16) + x * 128;   // S_x; P_x goes over its first 64 columns
     const uint32_t t_o = tmem + ((uint32_t)(wq * 32) << 16) + (NT + x) * 128;
     const float sl2 = p.scale_log2;
-    int n_s = 0, n_item = 0;
+    int n_s = 0, n_item = 0, n_out = 0;
     bool ok = true;
+    // all 128 threads of this warpgroup meet (bounded, like every other wait of the kernel)
+    auto meet = [&]() {
+      mbar_arrive(bar(C::BAR_OUT + x));
+      const bool m = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_OUT + x), (uint32_t)n_out & 1u, abort_flag, WAIT_LIMIT));
+      ++n_out;
+      return m;
+    };
     for (int i = first; i < p.n_items && ok; i += stride, ++n_item) {
       const Item it = load_item<PAIR_TILES>(p, i);
       // this M-tile's share of the item, in registers (x is not a compile-time index)
@@ -439,6 +449,43 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       const bool valid = row < my_rows;
       __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) + ((int64_t)(my_row0 + row) * p.Hq + h) * HD;
       uint32_t a[32], b[32];
+      if (my_rows >= BM) {
+        // A whole tile of this sequence: the rows go out as two 128 x 64 blocks through shared memory and the copy
+        // engine (each thread writing its own 256-byte row with 16-byte stores took 3600 clocks per item: 4096
+        // half-sector writes through one load/store unit).  Thread (row r, 16-byte chunk c) writes chunk c ^ (r % 8)
+        // of its 128-byte line, the 128-byte swizzle the tensor map expects.
+        const uint32_t out = base + C::OFF_OUT + x * HALF;
+        const bool issuer = wq == 0 && lane == 0;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          tmem_ld_32x32(t_o + hh * 64, a);
+          tmem_ld_32x32(t_o + hh * 64 + 32, b);
+          tmem_wait_ld(a);
+          tmem_wait_ld(b);
+          uint32_t w[8][4];   // the thread's 64 columns as bf16, packed while the block's previous copy is still being read
+#pragma unroll
+          for (int c = 0; c < 8; ++c) {
+            uint32_t(&cur)[32] = (c & 4) ? b : a;
+            const int e = (c & 3) * 8;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              w[c][u] = pack_bf16(__uint_as_float(cur[e + 2 * u]) * inv, __uint_as_float(cur[e + 2 * u + 1]) * inv);
+          }
+          if (issuer) bulk_wait_read0();        // the block's previous copy has left shared memory
+          ok = meet();
+          if (!ok) break;
+#pragma unroll
+          for (int c = 0; c < 8; ++c)
+            st_shared_v4(out + (uint32_t)row * 128 + (uint32_t)((c ^ (row & 7)) << 4), w[c][0], w[c][1], w[c][2], w[c][3]);
+          fence_async_smem();
+          ok = meet();
+          if (!ok) break;
+          if (issuer) {
+            tma_store_3d(&map_o, out, hh * 64, h, my_row0);
+            bulk_commit();
+          }
+        }
+      } else {
       tmem_ld_32x32(t_o, a);
       tmem_wait_ld(a);
 #pragma unroll
@@ -459,11 +506,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         }
         if (q + 1 < 4) tmem_wait_ld(nxt);
       }
+      }
       if (valid && p.lse != nullptr) p.lse[(int64_t)h * p.total + my_row0 + row] = (m_ref + log2f(l)) * kLn2;
       tc_fence_before();   // the next item's first P V overwrites O_x; it is issued after this warp's next arrive on P_x
     }
   }
 
+  if (warp >= 4 && (warp & 3) == 0 && lane == 0) bulk_wait_all0();   // this thread's output copies have completed
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, (int32_t)EARN_ERR_TIMEOUT);
@@ -568,9 +617,9 @@ bool prefill_tc_supported(const PrefillArgs& a, int total_tokens) {
 
 cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int plan_entries, void* plan, int32_t* status_word,
                               cudaStream_t st) {
-  CUtensorMap mq, mk, mv;
+  CUtensorMap mq, mk, mv, mo;
   if (!make_map(&mq, a.q, a.Hq, total_tokens) || !make_map(&mk, a.k, a.Hkv, total_tokens) ||
-      !make_map(&mv, a.v, a.Hkv, total_tokens))
+      !make_map(&mv, a.v, a.Hkv, total_tokens) || !make_map(&mo, a.o, a.Hq, total_tokens))
     return cudaErrorInvalidValue;
   if (plan_entries <= 0) return cudaSuccess;
   const int rows = prefill_rows_per_entry(a.Hq, a.Hkv);
@@ -590,11 +639,11 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int plan_e
   if (pair_tiles) {
     e = ensure_dynamic_smem<prefill_tc_kernel<true>>(Cfg::SMEM_BYTES);
     if (e == cudaSuccess)
-      e = launch_pdl(prefill_tc_kernel<true>, dim3(grid), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, mq, mk, mv, p);
+      e = launch_pdl(prefill_tc_kernel<true>, dim3(grid), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, mq, mk, mv, mo, p);
   } else {
     e = ensure_dynamic_smem<prefill_tc_kernel<false>>(Cfg::SMEM_BYTES);
     if (e == cudaSuccess)
-      e = launch_pdl(prefill_tc_kernel<false>, dim3(grid), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, mq, mk, mv, p);
+      e = launch_pdl(prefill_tc_kernel<false>, dim3(grid), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, mq, mk, mv, mo, p);
   }
   note_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
