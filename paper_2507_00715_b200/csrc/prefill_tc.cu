@@ -15,7 +15,7 @@
 //              from tensor memory; after the last P V of an item it goes straight on to the first S of the next
 //   warps 4..  one softmax warpgroup per M-tile, one query row per thread: S_x from TMEM in 32-column chunks,
 //              online softmax in the log2 domain in ONE pass per tile (the reference maximum of the row is the one
-//              the earlier tiles left; the first tile of an item finds its own in a pass of its own), packed
+//              the earlier tiles left; the first tile of an item takes the maximum of its first 32 columns), packed
 //              fp32x2 arithmetic, P_x kept in registers until the reference is known to hold and then written as
 //              bf16 over the first 64 columns of S_x; the same warps normalise and store O_x when the item ends,
 //              while the tensor core already works on the next item
@@ -342,7 +342,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int n_chunks = diag ? wq + 1 : (!PAIR_TILES || j < my_diag) ? 4 : 0;
         uint32_t a[32], b[32], pk[4][16];
         // row maximum of the visible part of S_x(j), scaled into the log2 domain (a pass of its own over TMEM)
-        auto row_max = [&]() {
+        auto row_max_all = [&]() {
           float mx = -INFINITY;
           tmem_ld_32x32(t_s, a);
           if (n_chunks > 1) tmem_ld_32x32(t_s + 32, b);
@@ -374,7 +374,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
           }
           return mx * sl2;
         };
-        if (j == 0) m_ref = row_max();   // first tile of the item: the reference is its own row maximum
         // ---- P = 2^(S * scale - m_ref) as bf16 pairs (kept in registers until the reference is known to hold) and
         //      their row sum, in one pass.  The reference is the one earlier tiles left.  If this tile's sum of
         //      exponentials exceeds 2^8 some logit may have outgrown the reference by more than the threshold
@@ -384,10 +383,24 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         float ls0, ls1;
 #pragma unroll 1
         for (int attempt = 0;; ++attempt) {
-          const float neg_m = -m_ref;
           ls0 = ls1 = 0.f;
           tmem_ld_32x32(t_s, a);
           tmem_wait_ld(a);
+          if (j == 0 && attempt == 0) {
+            // First tile of an item: the reference is the largest visible logit among the row's first 32 keys (the
+            // start of the sequence; column 0 is visible to every row).  A later column that outgrows it by more
+            // than the threshold shows in the sum below and sends the tile through the redo path like any other.
+            // (A pass of its own over all 128 columns for the exact row maximum cost 26 us per 7B-class layer.)
+            float mx = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 32; c += 4) {
+              const bool d0 = diag && wq == 0;   // on the diagonal chunk column c counts for row `lane` iff c <= lane
+              mx = max3(mx, (d0 && c > lane) ? -INFINITY : __uint_as_float(a[c]), (d0 && c + 1 > lane) ? -INFINITY : __uint_as_float(a[c + 1]));
+              m1 = max3(m1, (d0 && c + 2 > lane) ? -INFINITY : __uint_as_float(a[c + 2]), (d0 && c + 3 > lane) ? -INFINITY : __uint_as_float(a[c + 3]));
+            }
+            m_ref = fmaxf(mx, m1) * sl2;
+          }
+          const float neg_m = -m_ref;
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             if (q < n_chunks) {
@@ -417,7 +430,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
           const bool grow = !(ls0 + ls1 <= 256.f);   // also catches a sum that overflowed
           if (attempt > 0 || !__any_sync(0xffffffffu, grow)) break;
           // S_x(j) was issued after P_x V of tile j-1, so the commit that signalled it covers that too: O_x is quiescent
-          const float mxs = row_max();
+          // the whole warp repeats the pass (the TMEM accesses are warp-wide), but only the rows that grew take a new
+          // reference: a row's result depends on its own logits alone, whatever its neighbours in the tile do
+          const float mx_all = row_max_all();   // every lane takes part in the loads
+          const float mxs = grow ? mx_all : m_ref;
           const float alpha = mxs > m_ref ? ex2(m_ref - mxs) : 1.f;
           m_ref = fmaxf(m_ref, mxs);
           l0 *= alpha;
