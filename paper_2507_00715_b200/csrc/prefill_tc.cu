@@ -44,11 +44,11 @@ constexpr long long WAIT_LIMIT = 2000000000LL;     // about one second of SM clo
 constexpr int NT = 2;   // M-tiles per work item
 
 struct Cfg {
-  static constexpr int NSTAGE = 4;                          // ring entries (K and V tiles alternate); five measured the same
+  static constexpr int NSTAGE = 3;                          // ring entries (K and V tiles alternate); four and five measured the same
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_RING = OFF_Q + NT * TILE;
-  static constexpr int OFF_OUT = OFF_RING + NSTAGE * TILE;  // per M-tile: one 128 x 64 bf16 block of O on its way out
-  static constexpr int OFF_BAR = OFF_OUT + NT * HALF;
+  static constexpr int OFF_OUT = OFF_RING + NSTAGE * TILE;  // per M-tile: the 128 x 128 bf16 tile of O on its way out
+  static constexpr int OFF_BAR = OFF_OUT + NT * TILE;
   static constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;   // + alignment slack
   static constexpr int TMEM_COLS = NT * 256;                // S_x (and P_x over it) at x*128, O_x at (NT + x)*128
   static constexpr int THREADS = 32 * (4 + 4 * NT);
@@ -470,7 +470,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // engine (each thread writing its own 256-byte row with 16-byte stores took 3600 clocks per item: 4096
         // half-sector writes through one load/store unit).  Thread (row r, 16-byte chunk c) writes chunk c ^ (r % 8)
         // of its 128-byte line, the 128-byte swizzle the tensor map expects.
-        const uint32_t out = base + C::OFF_OUT + x * HALF;
+        const uint32_t out = base + C::OFF_OUT + x * TILE;
         const bool issuer = wq == 0 && lane == 0;
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
@@ -478,7 +478,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
           tmem_ld_32x32(t_o + hh * 64 + 32, b);
           tmem_wait_ld(a);
           tmem_wait_ld(b);
-          uint32_t w[8][4];   // the thread's 64 columns as bf16, packed while the block's previous copy is still being read
+          uint32_t w[8][4];   // the thread's 64 columns as bf16
 #pragma unroll
           for (int c = 0; c < 8; ++c) {
             uint32_t(&cur)[32] = (c & 4) ? b : a;
@@ -487,19 +487,23 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             for (int u = 0; u < 4; ++u)
               w[c][u] = pack_bf16(__uint_as_float(cur[e + 2 * u]) * inv, __uint_as_float(cur[e + 2 * u + 1]) * inv);
           }
-          if (issuer) bulk_wait_read0();        // the block's previous copy has left shared memory
-          ok = meet();
-          if (!ok) break;
+          if (hh == 0) {
+            if (issuer) bulk_wait_read0();      // the previous item's copies have left the staging tile (long ago)
+            ok = meet();
+            if (!ok) break;
+          }
 #pragma unroll
           for (int c = 0; c < 8; ++c)
-            st_shared_v4(out + (uint32_t)row * 128 + (uint32_t)((c ^ (row & 7)) << 4), w[c][0], w[c][1], w[c][2], w[c][3]);
+            st_shared_v4(out + hh * HALF + (uint32_t)row * 128 + (uint32_t)((c ^ (row & 7)) << 4), w[c][0], w[c][1], w[c][2], w[c][3]);
+        }
+        if (ok) {
           fence_async_smem();
           ok = meet();
-          if (!ok) break;
-          if (issuer) {
-            tma_store_3d(&map_o, out, hh * 64, h, my_row0);
-            bulk_commit();
-          }
+        }
+        if (ok && issuer) {
+          tma_store_3d(&map_o, out, 0, h, my_row0);
+          tma_store_3d(&map_o, out + HALF, 64, h, my_row0);
+          bulk_commit();
         }
       } else {
       tmem_ld_32x32(t_o, a);
