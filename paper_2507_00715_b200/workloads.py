@@ -148,8 +148,9 @@ def layer_qkv(w: Workload, layer: int, device="cpu") -> Tuple[torch.Tensor, torc
     q = _randn((total, w.n_q_heads, w.head_dim), _seed_for(w, "q", layer), device)
     k = _randn((total, w.n_kv_heads, w.head_dim), _seed_for(w, "k", layer), device)
     v = _randn((total, w.n_kv_heads, w.head_dim), _seed_for(w, "v", layer), device)
-    first = torch.as_tensor(cu[:-1].astype(np.int64), device=device)
-    last = torch.as_tensor((cu[1:] - 1).astype(np.int64), device=device)
+    has_rows = cu[1:] > cu[:-1]   # an empty sequence has no first or last row
+    first = torch.as_tensor(cu[:-1][has_rows].astype(np.int64), device=device)
+    last = torch.as_tensor((cu[1:] - 1)[has_rows].astype(np.int64), device=device)
     k[first] += 4.0 * u
     # a one-token sequence gets the bias once per role, as the recipe states it
     k[last] += 4.0 * u

@@ -137,6 +137,13 @@ def test_long_uneven_prompts_are_decoded_longest_first():
     run_workload_and_compare(w.replace(seed=29, beams=5), check_lse=False)
 
 
+def test_long_prompt_among_empty_ones():
+    """One long prompt and many empty ones (no registers): decode over an empty prompt cache sees the generated tokens
+    only, and the batch is too sparse for the longest-first table to fit the plan area, so the plain order is used."""
+    w = BASE.replace(seed=30, lens=(1100,) + (0,) * 69, batch=70, n_layers=1, split_k=1, r_head=0, r_tail=0, decode_steps=2)
+    run_workload_and_compare(w, check_lse=False)
+
+
 def test_a_wait_that_runs_out_is_reported_and_the_context_survives():
     """Failure detection without a fault: a bounded device-side wait on a barrier nothing completes gives up after
     its limit, the kernel returns normally with EARN_ERR_TIMEOUT in the status word, and the library keeps working."""
