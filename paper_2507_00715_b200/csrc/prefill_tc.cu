@@ -55,7 +55,7 @@ struct Cfg {
   // barriers
   static constexpr int BAR_FULL = 0, BAR_EMPTY = BAR_FULL + NSTAGE, BAR_QFULL = BAR_EMPTY + NSTAGE,
                        BAR_QFREE = BAR_QFULL + NT, BAR_S = BAR_QFREE + NT, BAR_P = BAR_S + NT, BAR_O = BAR_P + NT,
-                       BAR_OUT = BAR_O + NT, BAR_DRAIN = BAR_OUT + NT, N_BARS = BAR_DRAIN + 1;
+                       BAR_DRAIN = BAR_O + NT, N_BARS = BAR_DRAIN + 1;
   static_assert(8 * N_BARS + 16 <= 512, "barrier block");
 };
 
@@ -144,7 +144,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       mbar_init(bar(C::BAR_S + x), 1);
       mbar_init(bar(C::BAR_P + x), 128);
       mbar_init(bar(C::BAR_O + x), 1);
-      mbar_init(bar(C::BAR_OUT + x), 128);
     }
     mbar_init(bar(C::BAR_DRAIN), 1);
     *abort_flag = 0;
@@ -318,15 +317,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const uint32_t t_s = tmem + ((uint32_t)(wq * 32) << 16) + x * 128;   // S_x; P_x goes over its first 64 columns
     const uint32_t t_o = tmem + ((uint32_t)(wq * 32) << 16) + (NT + x) * 128;
     const float sl2 = p.scale_log2;
-    int n_s = 0, n_item = 0, n_out = 0;
+    int n_s = 0, n_item = 0;
     bool ok = true;
-    // all 128 threads of this warpgroup meet (bounded, like every other wait of the kernel)
-    auto meet = [&]() {
-      mbar_arrive(bar(C::BAR_OUT + x));
-      const bool m = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_OUT + x), (uint32_t)n_out & 1u, abort_flag, WAIT_LIMIT));
-      ++n_out;
-      return m;
-    };
     for (int i = first; i < p.n_items && ok; i += stride, ++n_item) {
       const Item it = load_item<PAIR_TILES>(p, i);
       // this M-tile's share of the item, in registers (x is not a compile-time index)
@@ -466,12 +458,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(p.o) + ((int64_t)(my_row0 + row) * p.Hq + h) * HD;
       uint32_t a[32], b[32];
       if (my_rows >= BM) {
-        // A whole tile of this sequence: the rows go out as two 128 x 64 blocks through shared memory and the copy
-        // engine (each thread writing its own 256-byte row with 16-byte stores took 3600 clocks per item: 4096
-        // half-sector writes through one load/store unit).  Thread (row r, 16-byte chunk c) writes chunk c ^ (r % 8)
-        // of its 128-byte line, the 128-byte swizzle the tensor map expects.
-        const uint32_t out = base + C::OFF_OUT + x * TILE;
-        const bool issuer = wq == 0 && lane == 0;
+        // A whole tile of this sequence goes out through shared memory and the copy engine (each thread writing its
+        // own 256-byte row with 16-byte stores took 3600 clocks per item: 4096 half-sector writes through one
+        // load/store unit).  Lane r of a warp writes 16-byte chunk c of its row at chunk c ^ (r % 8) of the row's
+        // 128-byte line, the 128-byte swizzle the tensor map expects.
+        // Each warp stages and sends its own 32 rows (two blocks of 32 x 64), so no warp waits for another.
+        const uint32_t out = base + C::OFF_OUT + x * TILE + (uint32_t)wq * (32 * 128);
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
           tmem_ld_32x32(t_o + hh * 64, a);
@@ -488,21 +480,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
               w[c][u] = pack_bf16(__uint_as_float(cur[e + 2 * u]) * inv, __uint_as_float(cur[e + 2 * u + 1]) * inv);
           }
           if (hh == 0) {
-            if (issuer) bulk_wait_read0();      // the previous item's copies have left the staging tile (long ago)
-            ok = meet();
-            if (!ok) break;
+            if (lane == 0) bulk_wait_read0();   // this warp's previous copies have left its staging rows (long ago)
+            __syncwarp();
           }
 #pragma unroll
           for (int c = 0; c < 8; ++c)
-            st_shared_v4(out + hh * HALF + (uint32_t)row * 128 + (uint32_t)((c ^ (row & 7)) << 4), w[c][0], w[c][1], w[c][2], w[c][3]);
+            st_shared_v4(out + hh * HALF + (uint32_t)lane * 128 + (uint32_t)((c ^ (lane & 7)) << 4), w[c][0], w[c][1], w[c][2], w[c][3]);
         }
-        if (ok) {
-          fence_async_smem();
-          ok = meet();
-        }
-        if (ok && issuer) {
-          tma_store_3d(&map_o, out, 0, h, my_row0);
-          tma_store_3d(&map_o, out + HALF, 64, h, my_row0);
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_3d(&map_o, out, 0, h, my_row0 + wq * 32);
+          tma_store_3d(&map_o, out + HALF, 64, h, my_row0 + wq * 32);
           bulk_commit();
         }
       } else {
@@ -532,7 +521,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     }
   }
 
-  if (warp >= 4 && (warp & 3) == 0 && lane == 0) bulk_wait_all0();   // this thread's output copies have completed
+  if (warp >= 4 && lane == 0) bulk_wait_all0();   // this thread's output copies have completed
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) atomicExch(p.status, (int32_t)EARN_ERR_TIMEOUT);
@@ -595,12 +584,12 @@ PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   return fn;
 }
 
-bool make_map(CUtensorMap* map, const void* ptr, int heads, int total) {
+bool make_map(CUtensorMap* map, const void* ptr, int heads, int total, int box_rows = BM) {
   auto fn = encode_fn();
   if (fn == nullptr) return false;
   cuuint64_t dims[3] = {(cuuint64_t)HD, (cuuint64_t)heads, (cuuint64_t)total};
   cuuint64_t strides[2] = {(cuuint64_t)HD * 2, (cuuint64_t)heads * HD * 2};
-  cuuint32_t box[3] = {64, 1, (cuuint32_t)BM};
+  cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
   cuuint32_t estr[3] = {1, 1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -639,7 +628,7 @@ cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int plan_e
                               cudaStream_t st) {
   CUtensorMap mq, mk, mv, mo;
   if (!make_map(&mq, a.q, a.Hq, total_tokens) || !make_map(&mk, a.k, a.Hkv, total_tokens) ||
-      !make_map(&mv, a.v, a.Hkv, total_tokens) || !make_map(&mo, a.o, a.Hq, total_tokens))
+      !make_map(&mv, a.v, a.Hkv, total_tokens) || !make_map(&mo, a.o, a.Hq, total_tokens, 32))   // O leaves in slabs of 32 rows, one per warp
     return cudaErrorInvalidValue;
   if (plan_entries <= 0) return cudaSuccess;
   const int rows = prefill_rows_per_entry(a.Hq, a.Hkv);
