@@ -464,28 +464,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // 128-byte line, the 128-byte swizzle the tensor map expects.
         // Each warp stages and sends its own 32 rows (two blocks of 32 x 64), so no warp waits for another.
         const uint32_t out = base + C::OFF_OUT + x * TILE + (uint32_t)wq * (32 * 128);
+        // 32-column chunks, the next one in flight while this one is scaled, packed and staged
+        if (lane == 0) bulk_wait_read0();   // this warp's previous copies have left its staging rows (long ago)
+        tmem_ld_32x32(t_o, a);
+        tmem_wait_ld(a);
+        __syncwarp();
 #pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-          tmem_ld_32x32(t_o + hh * 64, a);
-          tmem_ld_32x32(t_o + hh * 64 + 32, b);
-          tmem_wait_ld(a);
-          tmem_wait_ld(b);
-          uint32_t w[8][4];   // the thread's 64 columns as bf16
+        for (int q = 0; q < 4; ++q) {
+          uint32_t(&cur)[32] = (q & 1) ? b : a;
+          uint32_t(&nxt)[32] = (q & 1) ? a : b;
+          if (q + 1 < 4) tmem_ld_32x32(t_o + (q + 1) * 32, nxt);
 #pragma unroll
-          for (int c = 0; c < 8; ++c) {
-            uint32_t(&cur)[32] = (c & 4) ? b : a;
-            const int e = (c & 3) * 8;
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-              w[c][u] = pack_bf16(__uint_as_float(cur[e + 2 * u]) * inv, __uint_as_float(cur[e + 2 * u + 1]) * inv);
+          for (int c = 0; c < 4; ++c) {   // chunk c of this quarter = 16-byte chunk (q % 2) * 4 + c of block q / 2
+            const uint32_t w0 = pack_bf16(__uint_as_float(cur[c * 8 + 0]) * inv, __uint_as_float(cur[c * 8 + 1]) * inv);
+            const uint32_t w1 = pack_bf16(__uint_as_float(cur[c * 8 + 2]) * inv, __uint_as_float(cur[c * 8 + 3]) * inv);
+            const uint32_t w2 = pack_bf16(__uint_as_float(cur[c * 8 + 4]) * inv, __uint_as_float(cur[c * 8 + 5]) * inv);
+            const uint32_t w3 = pack_bf16(__uint_as_float(cur[c * 8 + 6]) * inv, __uint_as_float(cur[c * 8 + 7]) * inv);
+            const int ch = (q & 1) * 4 + c;
+            st_shared_v4(out + (q >> 1) * HALF + (uint32_t)lane * 128 + (uint32_t)((ch ^ (lane & 7)) << 4), w0, w1, w2, w3);
           }
-          if (hh == 0) {
-            if (lane == 0) bulk_wait_read0();   // this warp's previous copies have left its staging rows (long ago)
-            __syncwarp();
-          }
-#pragma unroll
-          for (int c = 0; c < 8; ++c)
-            st_shared_v4(out + hh * HALF + (uint32_t)lane * 128 + (uint32_t)((c ^ (lane & 7)) << 4), w[c][0], w[c][1], w[c][2], w[c][3]);
+          if (q + 1 < 4) tmem_wait_ld(nxt);
         }
         fence_async_smem();
         __syncwarp();
