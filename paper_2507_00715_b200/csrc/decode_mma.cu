@@ -14,8 +14,8 @@
 // straight from k_new / v_new, which split 0 also appends to the private segment).
 //
 // The list is cut into tiles of 16 positions.  The warp fetches them with 16-byte cp.async copies into
-// padded shared-memory tiles (a ring of four stages = 35 KB at head_dim 128, so six CTAs share an SM; two
-// stages for lists of at most two tiles).  Tile size, warps per CTA and ring depth were swept on B200 at
+// padded shared-memory tiles (a ring of four stages = 35 KB at head_dim 128, so six CTAs share an SM; three
+// stages, the whole list in flight at once, for lists of at most two tiles).  Tile size, warps per CTA and ring depth were swept on B200 at
 // the 7B shapes: (16, 1, 4) gave 50.9 us per layer against 51.3-63.4 us for the other combinations.
 // A long list is then consumed two tiles at a time (one softmax step, one rescale of the accumulator and one
 // round of quad shuffles per 32 positions, four independent MMA chains instead of two): 49.6 -> 46.3 us per

@@ -17,8 +17,9 @@
 //              online softmax in the log2 domain in ONE pass per tile (the reference maximum of the row is the one
 //              the earlier tiles left; the first tile of an item takes the maximum of its first 32 columns), packed
 //              fp32x2 arithmetic, P_x kept in registers until the reference is known to hold and then written as
-//              bf16 over the first 64 columns of S_x; the same warps normalise and store O_x when the item ends,
-//              while the tensor core already works on the next item
+//              bf16 over the first 64 columns of S_x; the same warps normalise O_x when the item ends, stage their
+//              32 rows each in shared memory and hand them to the copy engine (TMA store), while the tensor core
+//              already works on the next item
 // With two M-tiles the tensor core works on one while the other is in its softmax (S_A, S_B, O_A, O_B fill
 // the 512 TMEM columns).  The running output stays in TMEM.  The softmax reference maximum is only raised
 // when a tile's sum of exponentials exceeds 2^8 (no term can exceed that bound otherwise); then the owning warp
