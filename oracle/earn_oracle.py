@@ -17,11 +17,15 @@ What pins each function (see tests/test_oracle_pins.py):
   register_attention    : form A (gathered, Section 3.2 inference) must equal
                           form B (masked full-length, Section 3.2 training rule)
   DecodeState / decode_attention : step s equals the last row of a causal prefill
-                          over prompt ++ generated; W beams equal W independent runs
+                          over prompt ++ generated; W beams equal W independent runs;
+                          the sampled-row form of step() leaves the same cache and the
+                          same values on the selected rows as the plain form
   kv_entries, gamma_cache, gamma_attn, speedup : the worked example of Section 3.3
   rms_norm, apply_rope, register_qkv : closed forms (constant rows, zero angle, norm preservation), the
                           relative-position property of the rotation, a library rms_norm / linear call, and
                           "project every row then gather" = "gather then project" (Eq. 2 acts per token)
+  rope_tables           : closed-form angles (D = 8, theta = 10000: 1, 0.1, 0.01, 0.001 rad per position)
+  attention_scores, sparsity, sinks : the scalar definitions of Eq. 14-15 by hand
 Attention values have no printed worked example in the paper, so beyond those
 pins they are parity unpinned.
 """

@@ -381,3 +381,68 @@ def test_register_qkv_matches_library_ops_and_commutes_with_the_gather():
     x2[~keep] = rng.standard_normal((int((~keep).sum()), dm))
     q2, k2, v2 = orc.register_qkv(x2, cu, idx, wn, w, hq, hkv, d, cos, sin, eps=1e-6)
     assert np.array_equal(q, q2) and np.array_equal(k, k2) and np.array_equal(v, v2)
+
+
+# ---------------------------------------------------------------- sampled-row decode, rotary frequencies, scores
+def test_decode_step_with_sampled_rows_equals_the_plain_step():
+    """The sampled-row form of DecodeState.step (used where a workload is too large to compute in full) must keep
+    the cache exactly as the plain step does -- every beam appended and re-parented, selected or not -- and return
+    the plain step's values on the selected rows, zeros elsewhere (Eq. 4; Section 3.2 decoding rule)."""
+    rng = np.random.default_rng(11)
+    B, W, R, hq, hkv, d, T = 2, 3, 5, 4, 2, 4, 4
+    kc = [rng.standard_normal((R, hkv, d)) for _ in range(B)]
+    vc = [rng.standard_normal((R, hkv, d)) for _ in range(B)]
+    full, part = orc.DecodeState(kc, vc, W), orc.DecodeState(kc, vc, W)
+    for s in range(T):
+        dq = rng.standard_normal((B * W, hq, d))
+        dk = rng.standard_normal((B * W, hkv, d))
+        dv = rng.standard_normal((B * W, hkv, d))
+        parents = None if s == 0 else rng.integers(0, W, size=B * W)
+        # a different selection every step, so that a beam skipped at one step is read (through a child) at a later one
+        rows = {(int(j), int(h)) for j, h in zip(rng.integers(0, B * W, size=4), rng.integers(0, hq, size=4))}
+        o_full = full.step(dq, dk, dv, parents)
+        o_part = part.step(dq, dk, dv, parents, rows=rows)
+        for j in range(B * W):
+            for h in range(hq):
+                if (j, h) in rows:
+                    assert np.array_equal(o_part[j, h], o_full[j, h])
+                else:
+                    assert not o_part[j, h].any()
+        for j in range(B * W):
+            assert len(part.priv_k[j]) == len(full.priv_k[j]) == s + 1
+            assert np.array_equal(np.stack(part.priv_k[j]), np.stack(full.priv_k[j]))
+            assert np.array_equal(np.stack(part.priv_v[j]), np.stack(full.priv_v[j]))
+        assert [part.entries(b) for b in range(B)] == [full.entries(b) for b in range(B)] == [R + s + 1] * B
+    # and the selected rows are right by themselves: one of them against the scalar brute force
+    j, h = next(iter(rows))
+    keys = np.concatenate([kc[j // W][:, h // 2], np.stack(full.priv_k[j])[:, h // 2]])
+    vals = np.concatenate([vc[j // W][:, h // 2], np.stack(full.priv_v[j])[:, h // 2]])
+    ref = brute_attention_row(list(dq[j, h]), [list(x) for x in keys], [list(x) for x in vals], 0.5)
+    np.testing.assert_allclose(o_part[j, h], ref, atol=1e-13)
+
+
+def test_rope_frequency_ladder_closed_form():
+    """Pair i turns by pos * theta^(-2i/D): with D = 8 and theta = 10000 the four pairs turn by 1, 0.1, 0.01 and
+    0.001 radians per position (any other exponent on the ladder fails here)."""
+    cos, sin = orc.rope_tables(8, 8, theta=10000.0)
+    for pos in (1, 5):
+        np.testing.assert_allclose(cos[pos], np.cos(pos * np.array([1.0, 0.1, 0.01, 0.001])), atol=1e-15)
+        np.testing.assert_allclose(sin[pos], np.sin(pos * np.array([1.0, 0.1, 0.01, 0.001])), atol=1e-15)
+    # D = 4, theta = 16: pairs turn by 1 and 16^(-1/2) = 0.25 radians per position
+    cos, sin = orc.rope_tables(3, 4, theta=16.0)
+    np.testing.assert_allclose(sin[2], [math.sin(2.0), math.sin(0.5)], atol=1e-15)
+    # the pair (i, i + D/2) is what turns: unit vector on coordinate 1 of D = 8 moves into coordinate 5
+    r = orc.apply_rope(np.array([0.0, 1, 0, 0, 0, 0, 0, 0]), *(t[1] for t in orc.rope_tables(2, 8)))
+    np.testing.assert_allclose([r[1], r[5]], [math.cos(0.1), math.sin(0.1)], atol=1e-15)
+    assert not r[[0, 2, 3, 4, 6, 7]].any()
+
+
+def test_attention_scores_by_hand():
+    """Eq. 14-15 take the softmax scores of one row: compare with the scalar definition."""
+    rng = np.random.default_rng(12)
+    qrow, keys = rng.standard_normal(6), rng.standard_normal((7, 6))
+    p = orc.attention_scores(qrow, keys)
+    logits = [math.fsum(qrow[d] * keys[j][d] for d in range(6)) / math.sqrt(6) for j in range(7)]
+    z = math.fsum(math.exp(s) for s in logits)
+    np.testing.assert_allclose(p, [math.exp(s) / z for s in logits], atol=1e-15)
+    assert abs(p.sum() - 1.0) < 1e-15
