@@ -160,8 +160,8 @@ earn_status_t earn_register_qkv(const earn_model_t* model, const earn_batch_t* b
                                 void* workspace, size_t workspace_bytes, earn_stream_t stream);
 
 /* Step 3 — attention of a layer l >= k during prefill: causal attention among the R register tokens of
- * each sequence in the order [prefix; suffix] (Section 3.2, training rule "only register ... tokens
- * participate", and the inference rule above).  q_reg, o_reg: device [B, R, Hq, D]. */
+ * each sequence in the order [prefix; suffix] (Section 3.2: in layers l >= k only register and generated tokens
+ * attend, by the training rule and by the inference rule above).  q_reg, o_reg: device [B, R, Hq, D]. */
 earn_status_t earn_register_attn(const earn_model_t* model, const earn_batch_t* batch, int32_t layer,
                                  const void* q_reg, const earn_cache_t* cache, void* o_reg,
                                  void* workspace, size_t workspace_bytes, earn_stream_t stream);
@@ -195,7 +195,10 @@ earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* ba
  *     every call); make that first call outside any stream capture.
  *   - All calls on a device share the one array, which keeps the previous call's contents; each call clears
  *     the part that must start at zero on `stream` before its kernel.  Two calls that overlap on the GPU (different
- *     streams without an ordering between them) race on the array: serialise them. */
+ *     streams without an ordering between them) race on the array: serialise them.
+ *   - The array's status block is cleared by every call and the caller holds no pointer to it, so earn_device_status
+ *     cannot be used with this entry point (the decode kernels have no bounded waits to report).
+ *   - The argument checks of earn_decode_attn run first, on the host; a rejected call has touched nothing. */
 #define EARN_STATIC_SCRATCH_BYTES (8u << 20)
 earn_status_t earn_decode_attn_static(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, int32_t step,
                                       const void* q, const void* k_new, const void* v_new,

@@ -316,7 +316,7 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, int max_shared_len, cudaStrea
   const int max_tiles = (max_shared_len + beams_per_tile * a.step + KT - 1) / KT;
   const long ctas = (long)(a.plan.n_splits > 0 ? a.plan.n_splits : 1) * a.plan.row_tiles * a.Hkv * a.batch;
   const bool unsplit = a.plan.n_splits <= 1;
-  const bool four_warps = unsplit && max_tiles <= 16 && ctas < 148;
+  const bool four_warps = unsplit && max_tiles <= 16 && ctas < sm_count();
   // a list of one or two tiles goes into a three-stage ring whole; anything longer is walked in pairs
   const bool two_tiles = unsplit && max_tiles <= 2;
   if (a.D == 64)

@@ -210,7 +210,7 @@ cudaError_t launch_decode_rows(const DecodeArgs& a, cudaStream_t st) {
   // heads x 20 beams (768 CTAs): 26.7 -> 17.5 us per compact-cache layer, 42.4 -> 30.8 us per prompt-cache layer;
   // with few CTAs (8 long sequences, split) the deeper ring is the faster one, 49.8 against 54.0 us.
   const long ctas = (long)a.Hkv * (a.plan.n_splits > 0 ? a.plan.n_splits : 1) * a.batch;
-  const bool many = ctas > 4L * 148;
+  const bool many = ctas > 4L * sm_count();
   if (a.D == 64) return many ? launch_rows<64, 2, 4, 6>(a, st) : launch_rows<64, 2, 6, 4>(a, st);
   return many ? launch_rows<128, 2, 4, 6>(a, st) : launch_rows<128, 2, 6, 4>(a, st);
 }

@@ -49,7 +49,12 @@ extern "C" earn_status_t earn_decode_attn_static(const earn_model_t* model, cons
                                                  const void* k_full_or_null, const void* v_full_or_null,
                                                  const earn_cache_t* cache, void* o, earn_stream_t stream) {
   using namespace earn;
-  if (model == nullptr || batch == nullptr || cache == nullptr || cache->beams < 1) return EARN_ERR_INVALID_ARG;
+  // The ordinary decode call's argument checks come first: a bad model or batch must be turned away on the host
+  // before its fields are used to size anything, and a rejected call must not have enqueued the clearing below.
+  bool nothing_to_do = false;
+  const earn_status_t checked = validate_decode(model, batch, layer, step, q, k_new, v_new, k_full_or_null,
+                                                v_full_or_null, cache, o, &nothing_to_do);
+  if (checked != EARN_OK || nothing_to_do) return checked;
   // the same layout earn_decode_attn expects from a caller's workspace: status block, split tickets, split partials
   const size_t need = earn_workspace_bytes(model, batch, cache->beams);
   if (need > (size_t)EARN_STATIC_SCRATCH_BYTES) return EARN_ERR_WORKSPACE;   // this batch needs more than the built-in scratch

@@ -10,6 +10,17 @@ namespace earn {
 static std::atomic<uint64_t> g_launches{0};
 void note_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
+int sm_count() {
+  static std::atomic<int> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return kDefaultSms; }
+  if (dev >= 0 && dev < 64 && cached[dev].load(std::memory_order_relaxed) > 0) return cached[dev].load(std::memory_order_relaxed);
+  int n = 0;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) { (void)cudaGetLastError(); return kDefaultSms; }
+  if (dev >= 0 && dev < 64) cached[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
+
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -64,7 +75,7 @@ DecodePlan make_decode_plan(const earn_model_t& m, const earn_batch_t& b, int be
 #ifndef EARN_DECODE_SLOTS_PER_SM
 #define EARN_DECODE_SLOTS_PER_SM 4
 #endif
-  const long slots = (long)EARN_DECODE_SLOTS_PER_SM * 148;
+  const long slots = (long)EARN_DECODE_SLOTS_PER_SM * sm_count();
   long splits = slots / units;
   long max_splits = (max_shared_len + 63) / 64;
   if (splits > max_splits) splits = max_splits;
@@ -119,6 +130,33 @@ static KeySource paged_source(const earn_batch_t* b, const earn_cache_t* c) {
   s.block_table = c->block_table; s.pages_per_seq = c->pages_per_seq; s.n_pages = c->n_pages;
   s.paged = 1; s.n_regs = b->n_head_reg + b->n_tail_reg;
   return s;
+}
+
+// Every host-side check of a decode call except the workspace's (shared by earn_decode_attn and
+// earn_decode_attn_static, which must run them before it touches its scratch array).
+earn_status_t validate_decode(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, int32_t step,
+                              const void* q, const void* k_new, const void* v_new, const void* k_full,
+                              const void* v_full, const earn_cache_t* cache, const void* o, bool* nothing_to_do) {
+  *nothing_to_do = false;
+  earn_status_t s = check_model(model);
+  if (s != EARN_OK) return s;
+  s = check_batch(batch);
+  if (s != EARN_OK) return s;
+  if (layer < 0 || layer >= model->n_layers || cache == nullptr) return EARN_ERR_INVALID_ARG;
+  if (cache->beams < 1 || cache->max_new < 1 || step < 1 || step > cache->max_new) return EARN_ERR_INVALID_ARG;
+  if ((int64_t)batch->batch * cache->beams > 65535) return EARN_ERR_UNSUPPORTED;
+  if (batch->batch == 0) { *nothing_to_do = true; return EARN_OK; }
+  if (layer < model->split_k) {
+    if (!k_full || !v_full || !aligned16(k_full) || !aligned16(v_full)) return EARN_ERR_INVALID_ARG;
+  } else {
+    s = check_cache_shared(model, batch, cache);
+    if (s != EARN_OK) return s;
+  }
+  if (!q || !k_new || !v_new || !o || !cache->k_priv || !cache->v_priv) return EARN_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(o) || !aligned16(cache->k_priv) ||
+      !aligned16(cache->v_priv))
+    return EARN_ERR_INVALID_ARG;
+  return EARN_OK;
 }
 
 }  // namespace earn
@@ -280,26 +318,11 @@ earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* ba
                                const void* q, const void* k_new, const void* v_new, const void* k_full_or_null,
                                const void* v_full_or_null, const earn_cache_t* cache, void* o, void* workspace,
                                size_t workspace_bytes, earn_stream_t stream) {
-  earn_status_t s = check_model(model);
-  if (s != EARN_OK) return s;
-  s = check_batch(batch);
-  if (s != EARN_OK) return s;
-  if (layer < 0 || layer >= model->n_layers || cache == nullptr) return EARN_ERR_INVALID_ARG;
-  if (cache->beams < 1 || cache->max_new < 1 || step < 1 || step > cache->max_new) return EARN_ERR_INVALID_ARG;
-  if ((int64_t)batch->batch * cache->beams > 65535) return EARN_ERR_UNSUPPORTED;
-  if (batch->batch == 0) return EARN_OK;
+  bool nothing_to_do = false;
+  earn_status_t s = validate_decode(model, batch, layer, step, q, k_new, v_new, k_full_or_null, v_full_or_null, cache, o,
+                                    &nothing_to_do);
+  if (s != EARN_OK || nothing_to_do) return s;
   const bool early = layer < model->split_k;
-  if (early) {
-    if (!k_full_or_null || !v_full_or_null || !aligned16(k_full_or_null) || !aligned16(v_full_or_null))
-      return EARN_ERR_INVALID_ARG;
-  } else {
-    s = check_cache_shared(model, batch, cache);
-    if (s != EARN_OK) return s;
-  }
-  if (!q || !k_new || !v_new || !o || !cache->k_priv || !cache->v_priv) return EARN_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(o) || !aligned16(cache->k_priv) ||
-      !aligned16(cache->v_priv))
-    return EARN_ERR_INVALID_ARG;
   if (workspace == nullptr || !aligned16(workspace) || workspace_bytes < workspace_need(model, batch, cache->beams))
     return EARN_ERR_WORKSPACE;
 

@@ -53,7 +53,15 @@ size_t prefill_plan_bytes(const earn_batch_t& b);
 // status block + plan + tickets: the part of the workspace that must read zero before the first call
 size_t workspace_head_bytes(const earn_model_t& m, const earn_batch_t& b, int beams);
 
-void note_launch(int n = 1);   // host-side count of kernels launched by this library
+// host-side argument checks of a decode call (everything but the workspace); *nothing_to_do: valid call, empty batch
+earn_status_t validate_decode(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, int32_t step,
+                              const void* q, const void* k_new, const void* v_new, const void* k_full,
+                              const void* v_full, const earn_cache_t* cache, const void* o, bool* nothing_to_do);
+
+void note_launch(int n = 1);
+// SMs of the current device (queried once per device); kDefaultSms when no device can be asked (host-only sizing calls)
+constexpr int kDefaultSms = 148;
+int sm_count();   // host-side count of kernels launched by this library
 
 // Opt a kernel in to `bytes` of dynamic shared memory and the largest carveout, once per device (the attribute
 // calls are not free).

@@ -322,13 +322,6 @@ bool make_map_2d(CUtensorMap* map, const void* ptr, int rows, int cols, int box_
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int sm_count_qkv() {
-  int dev = 0, n = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return 1;
-  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 1;
-  return n;
-}
-
 template <int BN>
 cudaError_t launch_gemm(const RegisterQkvArgs& a, QkvParams p, int M, int N, int sms, cudaStream_t st) {
   CUtensorMap ma, mb;
@@ -360,7 +353,7 @@ cudaError_t launch_register_qkv(const RegisterQkvArgs& a, cudaStream_t st) {
   p.m_tiles = (M + BM - 1) / BM;
   // Two heads per tile unless that leaves most of the GPU idle: with few register rows (a batch of 24 prompts with
   // two registers each is ONE row tile) the layer is a stream of W_qkv, and one-head tiles put twice as many SMs on it.
-  const int sms = sm_count_qkv();
+  const int sms = sm_count();
   const bool narrow = (long)p.m_tiles * ((N + 255) / 256) * 3 <= 2L * sms;
   return narrow ? launch_gemm<128>(a, p, M, N, sms, st) : launch_gemm<256>(a, p, M, N, sms, st);
 }

@@ -6,7 +6,7 @@ from oracle import earn_oracle as orc
 from paper_2507_00715_b200 import workloads as wl
 from paper_2507_00715_b200.session import EarnSession
 
-# spec tolerances: bf16 inputs / fp32 accumulation, and the fp32 debug path
+# bf16 inputs with fp32 accumulation, and the fp32 debug path
 TOL = {"bf16": dict(max_abs=2e-2, mean_abs=2e-3), "f32": dict(max_abs=1e-5, mean_abs=1e-6)}
 
 

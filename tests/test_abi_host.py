@@ -106,6 +106,33 @@ def test_host_validation_compact_register_decode(lib):
     assert lib.earn_beam_reparent(2, 3, 4, 5, 0x1000, None, 0x2000, None) == B.EARN_ERR_INVALID_ARG
 
 
+def test_host_validation_decode_static(lib):
+    """The entry point with the built-in scratch runs the ordinary decode call's checks before it sizes or clears
+    anything: a malformed model must come back as an error code, not as a crash of the host process."""
+    b = FakeBatch([40, 50], 10, 10)
+    good = B.make_cache(0x1000, 0x1000, None, 2, 4, 0x1000, 0x1000, None, 1, 4, None)
+
+    def dec(model, layer=2, step=1, cache=good, q=0x1000, batch=b):
+        return lib.earn_decode_attn_static(C.byref(model), C.byref(batch.c), layer, step, q, 0x1000, 0x1000, None, None,
+                                           C.byref(cache), 0x1000, None)
+
+    n0 = lib.earn_launch_count()
+    m = B.make_model(4, 2, 8, 2, 128, "bf16")
+    assert dec(B.make_model(4, 2, 8, 0, 128, "bf16")) == B.EARN_ERR_INVALID_ARG     # no kv heads: no division by zero
+    assert dec(B.make_model(4, 2, 8, 3, 128, "bf16")) == B.EARN_ERR_INVALID_ARG     # Hq % Hkv
+    assert dec(B.make_model(4, 2, 8, 2, 96, "bf16")) == B.EARN_ERR_UNSUPPORTED
+    assert dec(m, step=0) == B.EARN_ERR_INVALID_ARG
+    assert dec(m, step=5) == B.EARN_ERR_INVALID_ARG
+    assert dec(m, layer=4) == B.EARN_ERR_INVALID_ARG
+    assert dec(m, layer=0) == B.EARN_ERR_INVALID_ARG                                 # a full layer needs the prompt K/V
+    assert dec(m, q=0) == B.EARN_ERR_INVALID_ARG
+    assert dec(m, q=0x1008) == B.EARN_ERR_INVALID_ARG
+    assert dec(m, cache=B.make_cache(0x1000, 0x1000, None, 1, 4, 0x1000, 0x1000, None, 1, 4, None)) == B.EARN_ERR_INVALID_ARG
+    assert dec(m, cache=B.make_cache(0x1000, 0x1000, None, 2, 4, 0x1000, 0x1000, None, 0, 4, None)) == B.EARN_ERR_INVALID_ARG
+    assert dec(m, batch=FakeBatch([], 0, 0, max_seqlen=0)) == B.EARN_OK               # empty batch: nothing to do
+    assert lib.earn_launch_count() == n0
+
+
 def test_host_validation_register_qkv(lib):
     m = B.make_model(4, 2, 8, 2, 128, "bf16")
     b = FakeBatch([40, 50], 10, 10)

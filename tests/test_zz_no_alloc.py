@@ -1,10 +1,12 @@
-"""The decode entry point that allocates nothing (earn_decode_attn_static) against the ordinary one.
+"""The decode entry point that allocates nothing (earn_decode_attn_static) against the ordinary one and the oracle.
 
 Collected last on purpose: a run that stops at the first failure has then already been through every other test.
 The caller this entry point exists for cannot allocate device memory (its host owns the memory pool, or it
 cannot afford cudaMalloc's synchronisation), so the library brings a fixed scratch array of its own.  The test
 passes the same inputs to both entry points, through the C ABI, and expects the same outputs, twice in a row,
-because the scratch array is shared by all calls and keeps what the previous call left in it.
+because the scratch array is shared by all calls and keeps what the previous call left in it.  The static call's
+output is also held against the CPU oracle's decode step, so the test stands without the ordinary entry point,
+and the device allocator's state is read before and after the static calls: it must not move.
 """
 import ctypes as C
 
@@ -12,41 +14,71 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import earn_oracle as orc
 from paper_2507_00715_b200 import binding as B
 from paper_2507_00715_b200 import workloads as wl
-from parity_util import TOL
+from parity_util import TOL, make_session, to_np
 
-
-def _session(w):
-    from parity_util import make_session
-    return make_session(w)
+SHAPES = {
+    # one long sequence and two kv heads: too few CTAs to fill the GPU unsplit, so the prompt-cache layer runs
+    # split-KV and the scratch memory (tickets + partials) is really used; one row tile
+    "split_one_row_tile": dict(batch=1, n_q_heads=8, n_kv_heads=2, lens=(2048,), beams=2),
+    # ten beams x group of 4 = 40 query rows per kv head: the several-row-tile kernel, split over the prompt
+    "split_several_row_tiles": dict(batch=1, n_q_heads=8, n_kv_heads=2, lens=(1536,), beams=10),
+    # two long prompts more than 1.25x apart: the longest-first order table is written into the scratch's plan area
+    "ragged_order_table": dict(batch=2, n_q_heads=8, n_kv_heads=2, lens=(1100, 2300), beams=1),
+}
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("shape", sorted(SHAPES))
 @pytest.mark.parametrize("early_layer", [True, False])
-def test_static_scratch_decode_matches_workspace_decode(early_layer):
-    # one long sequence and two kv heads: too few CTAs to fill the GPU unsplit, so the prompt-cache layer runs
-    # split-KV and the scratch memory (tickets + partials) is really used
-    w = wl.Workload("noalloc", batch=1, n_layers=2, split_k=1, n_q_heads=8, n_kv_heads=2, head_dim=128, dtype="bf16",
-                    prompt_len=0, lens=(2048,), r_head=16, r_tail=16, decode_steps=2, beams=2, seed=31)
-    ses = _session(w)
+def test_static_scratch_decode_matches_workspace_decode_and_oracle(early_layer, shape):
+    w = wl.Workload("noalloc", n_layers=2, split_k=1, head_dim=128, dtype="bf16", prompt_len=0, r_head=16, r_tail=16,
+                    decode_steps=2, seed=31, **SHAPES[shape])
+    ses = make_session(w)
     assert B.earn_workspace_bytes(ses.model, ses.batch, w.beams) <= B.STATIC_SCRATCH_BYTES
-    for layer in range(w.n_layers):
-        ses.prefill_layer(layer, *wl.layer_qkv(w, layer, "cuda"))
+    cu = wl.cu_seqlens(w)
+    idx = orc.register_indices(wl.seqlens(w), w.r_head, w.r_tail)
     layer = 0 if early_layer else 1
+    for l in range(w.n_layers):
+        q, k, v = wl.layer_qkv(w, l, "cuda")
+        ses.prefill_layer(l, q, k, v)
+        if l == layer:
+            kn, vn = to_np(k), to_np(v)
+            if early_layer:
+                shared = [kn[cu[b]:cu[b + 1]] for b in range(w.batch)], [vn[cu[b]:cu[b + 1]] for b in range(w.batch)]
+            else:
+                shared = list(orc.compact(kn, cu, idx)), list(orc.compact(vn, cu, idx))
+    state = orc.DecodeState(shared[0], shared[1], w.beams)
     tol = TOL[w.dtype]
-    for step in (1, 2):                                  # two calls in a row share the scratch array
+    # everything the loop needs is allocated before the allocator's state is read
+    steps = []
+    for step in (1, 2):
         q, k_new, v_new = wl.decode_qkv(w, layer, step, "cuda")
-        ref = torch.empty_like(q)
+        parents = wl.beam_parents(w, step) if w.beams > 1 and step > 1 else None
+        steps.append((step, q, k_new, v_new, parents, None if parents is None else torch.from_numpy(parents).cuda(),
+                      torch.empty_like(q), torch.full_like(q, float("nan"))))
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0 = torch.cuda.memory_allocated()
+    results = []
+    for step, q, k_new, v_new, parents, parents_dev, ref, got in steps:   # two calls in a row share the scratch array
+        ses.begin_step(step, parents_dev)
         B.earn_decode_attn(ses.model, ses.batch, layer, step, q, k_new, v_new, ses.cache(layer), ref,
                            ses.k_full[layer], ses.v_full[layer], ses.workspace)
-        got = torch.full_like(q, float("nan"))
         B.earn_decode_attn_static(ses.model, ses.batch, layer, step, q, k_new, v_new, ses.cache(layer), got,
                                   ses.k_full[layer], ses.v_full[layer])
         torch.cuda.synchronize()
-        err = (got.double() - ref.double()).abs()
+    assert torch.cuda.memory_allocated() == alloc0, "a tensor was allocated during the static calls"
+    assert torch.cuda.mem_get_info()[0] == free0, "device memory was taken or returned during the static calls"
+    for step, q, k_new, v_new, parents, parents_dev, ref, got in steps:
         assert torch.isfinite(got.float()).all()
+        err = (got.double() - ref.double()).abs()
         assert err.max().item() <= tol["max_abs"] and err.mean().item() <= tol["mean_abs"], (step, err.max().item())
+        want = state.step(to_np(q), to_np(k_new), to_np(v_new), parents)
+        err = np.abs(got.double().cpu().numpy() - want)
+        assert err.max() <= tol["max_abs"] and err.mean() <= tol["mean_abs"], ("oracle", step, err.max(), err.mean())
     assert ses.device_status() == 0
 
 
