@@ -29,14 +29,23 @@ METRIC = "EARN attn tokens/s/GPU (prefill+decode, 7B GQA)"
 UNIT = "tokens/s"
 
 
+# Datasheet figures of the part, for context beside the measured ones: dense bf16 tensor throughput and the HBM3e
+# bandwidth in its round form (the HGX board is specified at 7.7 TB/s).
+NOMINAL = dict(tflops=2250.0, hbm_gbs=8000.0)
+
+
 def read_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
             p = json.load(f)
-        return dict(hbm_gbs=p["hbm_gbs"], tflops_burst=p["bf16_tflops"], tflops_sustained=p["bf16_tflops_sustained"],
-                    source="measured")
-    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+        out = dict(hbm_gbs=p["hbm_gbs"], tflops_burst=p["bf16_tflops"], tflops_sustained=p["bf16_tflops_sustained"],
+                   source="measured")
+    else:
+        out = dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+    out.update(nominal_tflops=NOMINAL["tflops"], nominal_hbm_gbs=NOMINAL["hbm_gbs"],
+               note="frac = achieved / measured peak (burst for the tensor-bound kernel); frac_nominal = achieved / datasheet")
+    return out
 
 
 KERNEL_SOURCES = {"prefill": "prefill_tc.cu", "compact": "compact.cu", "register": "register_mma.cu", "register_qkv": "register_qkv.cu",
@@ -101,7 +110,10 @@ def algorithmic(w: wl.Workload):
     out = {}
     out["prefill"] = dict(flops=4.0 * D * Hq * float((lens * (lens + 1) // 2).sum()),
                           bytes=float(tot * D * es * (2 * Hq + 2 * Hkv)))
-    out["compact"] = dict(flops=0.0, bytes=float(2 * B * R * D * es * (2 * Hkv + Hq) + B * R * 4))
+    # compaction: the K and V register rows, read and written, plus the index list.  The gathered Q rows that
+    # earn_compact_kv can also write are this library's way of feeding earn_register_attn, not work the method asks
+    # for: they count as traffic, not as algorithmic bytes (the register layer's Q rows are counted once, below).
+    out["compact"] = dict(flops=0.0, bytes=float(2 * 2 * B * R * Hkv * D * es + B * R * 4))
     out["register"] = dict(flops=4.0 * D * Hq * B * R * (R + 1) / 2, bytes=float(B * R * D * es * (2 * Hq + 2 * Hkv)))
     # hidden-state form of a register layer: the projection of the B*R register rows (bf16 path only)
     M, N, K = B * R, (Hq + 2 * Hkv) * D, w.d_model
@@ -190,6 +202,12 @@ class GpuJob:
         self.o_dec = torch.empty(w.batch * w.beams, w.n_q_heads, w.head_dim, **kw)
         self.graphs = None
         self.marks = []
+
+    def device_status(self) -> int:
+        return self.ses.device_status()
+
+    def kv_entries(self, generated: int) -> int:
+        return self.ses.kv_entries(generated)
 
     # ---- the step as an ordered list of segments; each segment = consecutive launches of one kind
     def segments(self):
@@ -537,8 +555,66 @@ def blas_threads() -> int:
         return os.cpu_count() or 1
 
 
+def timed_oracle(sample: "OracleSample"):
+    """(wall seconds, cores the run kept busy, threads it could have used).  The oracle is numpy: its matrix
+    products go to a threaded BLAS, everything else runs on one thread, so the cores it really used are read off
+    the process's CPU time over the wall time of the run rather than off the BLAS pool size."""
+    c0, w0 = time.process_time(), time.perf_counter()
+    t = sample.run()
+    c1, w1 = time.process_time(), time.perf_counter()
+    busy = (c1 - c0) / max(w1 - w0, 1e-9)
+    return t, max(1, int(round(busy))), busy, blas_threads()
+
+
 # ------------------------------------------------------------------------------------------------
-def main():
+# timers: the GPU arm times with CUDA events on the launching stream; a CPU job (the launcher's test) with the
+# host clock
+# ------------------------------------------------------------------------------------------------
+class DeviceTimer:
+    def start(self):
+        self.e0, self.e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        self.e0.record()
+
+    def stop(self):
+        self.e1.record()
+
+    def seconds(self) -> float:
+        torch.cuda.synchronize()
+        return self.e0.elapsed_time(self.e1) * 1e-3
+
+
+class HostTimer:
+    def start(self):
+        self.t0 = time.perf_counter()
+
+    def stop(self):
+        self.t1 = time.perf_counter()
+
+    def seconds(self) -> float:
+        return self.t1 - self.t0
+
+
+def free_port() -> int:
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        return sock.getsockname()[1]
+
+
+def _rank_entry(local_rank: int, world: int, port: int, argv, backend: str, job_factory):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(local_rank), LOCAL_RANK=str(local_rank),
+                      WORLD_SIZE=str(world))
+    main(argv, backend=backend, job_factory=job_factory)
+
+
+def spawn_ranks(n: int, argv, backend: str = "nccl", job_factory=None) -> None:
+    """`bench.py --gpus N` started as ONE process: start N ranks of this program on this node, one per GPU (rank =
+    local rank = device index), rendezvous on 127.0.0.1, and wait for them.  Rank 0 prints the line."""
+    import torch.multiprocessing as mp
+    mp.spawn(_rank_entry, args=(n, free_port(), list(argv), backend, job_factory), nprocs=n, join=True)
+
+
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
@@ -547,6 +623,8 @@ def main():
     ap.add_argument("--split-k", type=int, default=None)
     ap.add_argument("--prompt-len", type=int, default=None, help="override the workload's prompt length (uniform)")
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch size")
+    ap.add_argument("--decode-steps", type=int, default=None,
+                    help="override the workload's decode steps T; 0 = the prefill-only operating point")
     ap.add_argument("--impl", default="earn", choices=["earn", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -558,12 +636,12 @@ def main():
     ap.add_argument("--sweep-k", default=None,
                     help="comma-separated split layers k: time the workload once per k (one JSON line each, k = N is the "
                          "vanilla model) instead of the single benchmark line")
-    args = ap.parse_args()
+    args = ap.parse_args(argv)
     args.warmup = max(args.warmup, 3) if args.impl == "earn" else args.warmup
+    return args
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+def pick_workload(args) -> wl.Workload:
     w = wl.CONFIGS[args.config]
     if args.split_k is not None:
         w = w.replace(split_k=args.split_k)
@@ -571,80 +649,117 @@ def main():
         w = w.replace(prompt_len=args.prompt_len, lens=())
     if args.batch is not None:
         w = w.replace(batch=args.batch)
+    if args.decode_steps is not None:
+        w = w.replace(decode_steps=args.decode_steps)
+    return w
+
+
+def reference_arm(args, w, config):
+    sample = OracleSample(w, None, layer_stride=4)   # about a second of oracle work per step
+    for _ in range(args.warmup):
+        sample.run()
+    runs = [timed_oracle(sample) for _ in range(args.steps)]
+    t = sum(r[0] for r in runs) / len(runs)
+    val = sample.tokens / t
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic", "config": config,
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": max(r[1] for r in runs), "kind": "oracle (numpy float64)",
+                         "sample": sample.desc, "cores_busy_mean": sum(r[2] for r in runs) / len(runs),
+                         "blas_threads_available": runs[0][3]},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+# ------------------------------------------------------------------------------------------------
+def main(argv=None, backend: str = "nccl", job_factory=None):
+    """One rank of the benchmark (or, for `--gpus N` without a launcher's environment, the parent that starts N).
+    job_factory(workload, device, rank) replaces the GPU job -- the launcher's CPU test passes a stand-in that
+    has no kernels to run; the rank logic (rendezvous, barrier, max over ranks, rank 0 prints) is the same."""
+    args = parse_args(argv)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "earn":
+        spawn_ranks(args.gpus, sys.argv[1:] if argv is None else argv, backend, job_factory)
+        return
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    w = pick_workload(args)
     lens = wl.seqlens(w)
     tokens_per_step = int(lens.sum()) + w.batch * w.beams * w.decode_steps
     config = {"workload": workload_desc(w), "l2": "per-layer inputs and caches exceed the 126 MB L2; no flush needed",
               "sharding": "every rank runs the whole batch of its own seed (no data-path collective)"}
 
     if args.impl == "reference":
-        if rank != 0:
-            return
-        sample = OracleSample(w, None, layer_stride=4)   # about a second of oracle work per step
-        for _ in range(args.warmup):
-            sample.run()
-        times = [sample.run() for _ in range(args.steps)]
-        t = sum(times) / len(times)
-        val = sample.tokens / t
-        print(json.dumps({
-            "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f64", "data": "synthetic", "config": config,
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample.desc},
-            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+        if rank == 0:
+            reference_arm(args, w, config)
         return
 
-    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
+    on_gpu = job_factory is None
+    if on_gpu:
+        assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+        torch.cuda.set_device(local_rank)
+        dev = torch.device("cuda", local_rank)
+    else:
+        dev = torch.device("cpu")
     dist = None
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-    import __graft_entry__ as entry
-    if local_rank == 0:
-        entry.build()
-    if dist is not None:
-        dist.barrier()
-    from paper_2507_00715_b200 import binding as B
+        if on_gpu:
+            dist.init_process_group(backend, device_id=dev)
+        else:
+            dist.init_process_group(backend, rank=rank, world_size=world)
+    B = None
+    if on_gpu:
+        import __graft_entry__ as entry
+        if local_rank == 0:
+            entry.build()
+        if dist is not None:
+            dist.barrier()
+        from paper_2507_00715_b200 import binding as B
 
-    if args.profile_kernel:
+    if on_gpu and args.profile_kernel:
         profile_one_kernel(w, dev, args.profile_kernel)
         return
 
-    if args.sweep_k:
+    if on_gpu and args.sweep_k:
         sweep_split_layer(w, dev, [int(x) for x in args.sweep_k.split(",")], args)
         return
 
-    job = GpuJob(replicas.rank_workload(w, rank), dev)
+    w_rank = replicas.rank_workload(w, rank)
+    job = GpuJob(w_rank, dev) if on_gpu else job_factory(w_rank, dev, rank)
     peaks = read_peaks()
 
     def barrier():
         if dist is not None:
             dist.barrier()
-        torch.cuda.synchronize()
+        if on_gpu:
+            torch.cuda.synchronize()
 
-    n0 = B.earn_launch_count()
+    n0 = B.earn_launch_count() if on_gpu else 0
     job.step()                                   # first pass: plain launches (also sets per-kernel attributes)
-    launches_per_step = B.earn_launch_count() - n0
-    torch.cuda.synchronize()
-    if not args.no_graphs:
-        job.capture_graphs()                     # the same launches, recorded once, replayed per step
+    launches_per_step = (B.earn_launch_count() - n0) if on_gpu else getattr(job, "launches_per_step", 0)
+    if on_gpu:
+        torch.cuda.synchronize()
+        if not args.no_graphs:
+            job.capture_graphs()                 # the same launches, recorded once, replayed per step
     for _ in range(args.warmup):
         job.step()
     barrier()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
+    sampler = ClockSampler(local_rank) if rank == 0 and on_gpu else None
+    timer = DeviceTimer() if on_gpu else HostTimer()
+    timer.start()
     for _ in range(args.steps):
         job.step(record=True)
-    e1.record()
+    timer.stop()
     barrier()
     launches = launches_per_step * args.steps
     clocks = sampler.stop() if sampler else None
-    elapsed = replicas.max_over_ranks(e0.elapsed_time(e1) * 1e-3, dist, dev)
-    assert job.ses.device_status() == 0, "a device-side wait timed out"
+    elapsed = replicas.max_over_ranks(timer.seconds(), dist, dev)
+    ranks_ran = replicas.count_ranks(dist, dev)
+    assert job.device_status() == 0, "a device-side wait timed out"
     t_step = elapsed / args.steps
-    value = replicas.job_throughput(tokens_per_step, world, t_step)
+    value = replicas.job_throughput(tokens_per_step, ranks_ran, t_step)
 
     # rooflines from the events recorded at the segment boundaries INSIDE the timed region
     alg = algorithmic(w)
@@ -660,24 +775,30 @@ def main():
     rooflines = {}
     for kind, (sec, per_step, share) in job.segment_times().items():
         a = alg[kind]
+        r = {"kernel": kind}
         if kind == "prefill":
-            ach, peak, unit, bound = a["flops"] / sec / 1e12, peaks["tflops_sustained"], "TFLOP/s", "tensor"
-            src = peaks["source"] + " (sustained bf16)"
+            # tensor-bound: the burst cuBLAS figure is the stricter denominator and the one `frac` uses; the
+            # sustained one (a seconds-long GEMM loop under the power cap) is printed beside it
+            ach = a["flops"] / sec / 1e12
+            r.update(bound="tensor", achieved=ach, peak=peaks["tflops_burst"], unit="TFLOP/s",
+                     frac=ach / peaks["tflops_burst"], frac_burst=ach / peaks["tflops_burst"],
+                     frac_sustained=ach / peaks["tflops_sustained"], peak_sustained=peaks["tflops_sustained"],
+                     frac_nominal=ach / NOMINAL["tflops"], peak_source=peaks["source"] + " (burst bf16 GEMM)")
         else:
-            ach, peak, unit, bound = a["bytes"] / sec / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
-            src = peaks["source"] + " (copy)"
+            ach = a["bytes"] / sec / 1e9
+            r.update(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
+                     frac_nominal=ach / NOMINAL["hbm_gbs"], peak_source=peaks["source"] + " (copy)")
         if kind == "register_layer":
             tr = traffic.get("compact", 0) + traffic.get("register", 0) if {"compact", "register"} <= set(traffic) else None
         else:
             tr = traffic.get(kind)
-        rooflines[kind] = {"kernel": kind, "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
-                           "peak_source": src, "traffic": tr, "avg_launch_ms": sec * 1e3,
-                           "launches_per_step": per_step, "share_of_step": share,
-                           "algorithmic_flops_per_launch": a["flops"], "algorithmic_bytes_per_launch": a["bytes"]}
+        r.update(traffic=tr, avg_launch_ms=sec * 1e3, launches_per_step=per_step, share_of_step=share,
+                 algorithmic_flops_per_launch=a["flops"], algorithmic_bytes_per_launch=a["bytes"])
+        rooflines[kind] = r
     roofline = max(rooflines.values(), key=lambda r: r["share_of_step"]) if rooflines else None
 
     parts = None
-    if not args.no_parts and rank == 0:
+    if on_gpu and not args.no_parts and rank == 0:
         tp = job.time_parts()
         parts = {}
         for name, sec in tp.items():
@@ -687,27 +808,27 @@ def main():
                            "traffic": traffic.get(name)}
 
     e2e = None
-    if not args.no_e2e:
+    if on_gpu and not args.no_e2e:
         h2d, d2h = job.setup_e2e()
         job.step_e2e()
         barrier()
         n_e2e = max(1, min(args.steps, 2))
-        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a0.record()
+        t2 = DeviceTimer()
+        t2.start()
         for _ in range(n_e2e):
             job.step_e2e()
-        a1.record()
+        t2.stop()
         barrier()
-        te = replicas.max_over_ranks(a0.elapsed_time(a1) * 1e-3 / n_e2e, dist, dev)
-        e2e = {"value": world * tokens_per_step / te, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+        te = replicas.max_over_ranks(t2.seconds() / n_e2e, dist, dev)
+        e2e = {"value": ranks_ran * tokens_per_step / te, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "ms_per_step": te * 1e3, "steps": n_e2e}
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if on_gpu and rank == 0 and world == 1 and not args.no_cpu_baseline:
         sample = OracleSample(w, job)
-        tc = sample.run()
-        cpu = {"value": sample.tokens / tc, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample.desc,
-               "seconds": tc}
+        tc, cores, busy, avail = timed_oracle(sample)
+        cpu = {"value": sample.tokens / tc, "unit": UNIT, "cores": cores, "kind": "oracle (numpy float64)",
+               "sample": sample.desc, "seconds": tc, "cores_busy_mean": busy, "blas_threads_available": avail}
 
     if rank == 0:
         T, N, k = w.decode_steps, w.n_layers, w.split_k
@@ -716,15 +837,22 @@ def main():
             t_prefill = k * parts.get("prefill", {}).get("ms_per_launch", 0) + (N - k) * (
                 parts.get("compact", {}).get("ms_per_launch", 0) + parts.get("register", {}).get("ms_per_launch", 0))
             extra["prefill_tokens_per_s_isolated"] = int(lens.sum()) / (t_prefill * 1e-3) if t_prefill else None
-        earn_e, van_e = job.ses.kv_entries(T), N * (int(lens.sum()) + w.batch * w.beams * T)
+        seg = {kind: r["avg_launch_ms"] * r["launches_per_step"] for kind, r in rooflines.items()}
+        t_pre = seg.get("prefill", 0.0) + seg.get("register_layer", 0.0)
+        t_dec = seg.get("decode_full", 0.0) + seg.get("decode_compact", 0.0)
+        if t_pre > 0:
+            extra["prefill_tokens_per_s"] = ranks_ran * int(lens.sum()) / (t_pre * 1e-3)
+        if t_dec > 0:
+            extra["decode_tokens_per_s"] = ranks_ran * w.batch * w.beams * T / (t_dec * 1e-3)
+        earn_e, van_e = job.kv_entries(T), N * (int(lens.sum()) + w.batch * w.beams * T)
         print(json.dumps({
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ranks_ran, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": t_step * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": w.dtype, "data": "synthetic", "config": config, "clocks": clocks, "e2e": e2e,
             "gpu_launches": int(launches), "roofline": roofline, "rooflines": rooflines, "cpu_baseline": cpu,
-            "launch_mode": "plain" if args.no_graphs else "cuda-graph replay, one graph per segment",
-            "sequences_per_s": world * w.batch / t_step, "kernels": parts, "kv_reduction": 1.0 - earn_e / van_e,
-            "peaks": peaks, **extra}))
+            "launch_mode": "plain" if args.no_graphs or not on_gpu else "cuda-graph replay, one graph per segment",
+            "sequences_per_s": ranks_ran * w.batch / t_step, "kernels": parts, "kv_reduction": 1.0 - earn_e / van_e,
+            "peaks": peaks, **extra}), flush=True)
     if dist is not None:
         dist.destroy_process_group()
 

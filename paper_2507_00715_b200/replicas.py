@@ -25,6 +25,16 @@ def max_over_ranks(seconds: float, dist=None, device="cpu") -> float:
     return float(t.item())
 
 
+def count_ranks(dist=None, device="cpu") -> int:
+    """How many ranks really took part (each contributes one to a sum over the process group)."""
+    if dist is None or not dist.is_initialized():
+        return 1
+    import torch
+    t = torch.ones(1, dtype=torch.int64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return int(t.item())
+
+
 def job_throughput(units_per_rank: int, world: int, seconds: float) -> float:
     """Whole-job units per second under weak scaling: every rank processed `units_per_rank` in `seconds`."""
     return world * units_per_rank / seconds

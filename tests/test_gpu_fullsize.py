@@ -102,6 +102,61 @@ def run_fullsize(w, decode_steps=2, n_random=1500, n_decode_rows=600):
     assert ses.device_status() == 0
 
 
+def run_layer_mix(w, n_random=300, n_decode_rows=80, decode_steps=2):
+    """Any number of layers on either side of the split: sampled prefill rows for the full layers, compaction in full and
+    register attention in full for the register layers, sampled decode rows for every layer."""
+    rng = np.random.Generator(np.random.Philox(w.seed + 1000 * w.split_k))
+    w = w.replace(decode_steps=decode_steps)
+    cu, lens = wl.cu_seqlens(w), wl.seqlens(w)
+    ses = make_session(w)
+    idx = orc.register_indices(lens, w.r_head, w.r_tail)
+    R = w.n_regs
+    states = []
+    for layer in range(w.n_layers):
+        q, k, v = wl.layer_qkv(w, layer, "cuda")
+        o = ses.prefill_layer(layer, q, k, v)
+        qn, kn, vn = to_np(q), to_np(k), to_np(v)
+        if layer < w.split_k:
+            tok, head = sampled_prefill_rows(w, cu, rng, n_random)
+            ref = orc.causal_attention_rows(qn, kn, vn, cu, tok, head)
+            got = o[torch.from_numpy(tok).cuda(), torch.from_numpy(head).cuda()].double().cpu().numpy()
+            check(got, ref, w.dtype, f"{w.name} k={w.split_k} prefill layer {layer}")
+            states.append(orc.DecodeState([kn[cu[b]:cu[b + 1]] for b in range(w.batch)],
+                                          [vn[cu[b]:cu[b + 1]] for b in range(w.batch)], w.beams))
+        else:
+            kc, vc, qc = orc.compact(kn, cu, idx), orc.compact(vn, cu, idx), orc.compact(qn, cu, idx)
+            assert np.array_equal(ses.reg_idx.cpu().numpy()[:, :R], idx)
+            ks = to_np(ses.k_shared[layer]).reshape(w.batch, ses.pages_per_seq * 16, w.n_kv_heads, w.head_dim)[:, :R]
+            vs = to_np(ses.v_shared[layer]).reshape(w.batch, ses.pages_per_seq * 16, w.n_kv_heads, w.head_dim)[:, :R]
+            assert ks.tobytes() == kc.tobytes() and vs.tobytes() == vc.tobytes(), f"compact cache, layer {layer}"
+            check(o.double().cpu().numpy(), orc.register_attention(qc, kc, vc), w.dtype,
+                  f"{w.name} k={w.split_k} register layer {layer}")
+            states.append(orc.DecodeState(list(kc), list(vc), w.beams))
+    n_beams = w.batch * w.beams
+    for step in range(1, decode_steps + 1):
+        pick_j = np.concatenate([[0, n_beams - 1], rng.integers(0, n_beams, size=n_decode_rows)])
+        pick_h = np.concatenate([[0, w.n_q_heads - 1], rng.integers(0, w.n_q_heads, size=n_decode_rows)])
+        rows = set(zip(pick_j.tolist(), pick_h.tolist()))
+        jj, hh = np.array([r[0] for r in rows]), np.array([r[1] for r in rows])
+        for layer in range(w.n_layers):
+            dq, dk, dv = wl.decode_qkv(w, layer, step, "cuda")
+            od = ses.decode_layer(layer, step, dq, dk, dv)
+            ref = states[layer].step(to_np(dq), to_np(dk), to_np(dv), None, rows=rows)
+            check(od.double().cpu().numpy()[jj, hh], ref[jj, hh], w.dtype,
+                  f"{w.name} k={w.split_k} decode step {step} layer {layer}")
+    assert ses.device_status() == 0
+    # Eq. 9 on the buffers the session really holds
+    earn, van = orc.kv_entries(lens, w.n_layers, w.split_k, R, generated=decode_steps)
+    assert ses.kv_entries(decode_steps) == earn and van == w.n_layers * (int(lens.sum()) + w.batch * decode_steps)
+
+
+@pytest.mark.parametrize("k", [0, 1, 2, 3, 4])
+def test_split_layer_sweep_on_long_history_shapes(k):
+    """The split sweep of the long-history workload changes which layers take which kernel: four layers of one
+    4096-token prompt at every split from k = 0 (registers only from the first layer) to k = N (vanilla model)."""
+    run_layer_mix(wl.CONFIGS["long"].replace(batch=1, n_layers=4, split_k=k))
+
+
 def test_fullsize_1p5b():
     run_fullsize(wl.CONFIGS["1p5b"])
 
