@@ -59,10 +59,20 @@ def test_static_scratch_decode_matches_workspace_decode_and_oracle(early_layer, 
         parents = wl.beam_parents(w, step) if w.beams > 1 and step > 1 else None
         steps.append((step, q, k_new, v_new, parents, None if parents is None else torch.from_numpy(parents).cuda(),
                       torch.empty_like(q), torch.full_like(q, float("nan"))))
+    # The set-up call: the first use of the entry point on a device looks up the scratch array's address, and the
+    # driver, which loads a module's code and data on first use, only now takes the array's 8 MiB (and the kernels'
+    # code) from device memory.  It is step 1 itself, which the loop below repeats with the same result.
+    step, q, k_new, v_new, _, _, ref, got = steps[0]
+    B.earn_decode_attn(ses.model, ses.batch, layer, step, q, k_new, v_new, ses.cache(layer), ref,
+                       ses.k_full[layer], ses.v_full[layer], ses.workspace)
+    B.earn_decode_attn_static(ses.model, ses.batch, layer, step, q, k_new, v_new, ses.cache(layer), got,
+                              ses.k_full[layer], ses.v_full[layer])
+    if steps[1][5] is not None:   # the re-parenting kernel of step 2 is loaded too (into a table the loop rewrites)
+        B.earn_beam_reparent(w.batch, w.beams, ses.max_new, 2, steps[1][5], None, ses.lineage[1])
+    got.fill_(float("nan"))
     torch.cuda.synchronize()
     free0, _ = torch.cuda.mem_get_info()
     alloc0 = torch.cuda.memory_allocated()
-    results = []
     for step, q, k_new, v_new, parents, parents_dev, ref, got in steps:   # two calls in a row share the scratch array
         ses.begin_step(step, parents_dev)
         B.earn_decode_attn(ses.model, ses.batch, layer, step, q, k_new, v_new, ses.cache(layer), ref,
