@@ -62,7 +62,17 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   using G = Geo<D>;
   constexpr int NTILES = D / 8, CH = G::CH, RPI = G::RPI, NIT = KT / RPI;
   extern __shared__ __align__(128) uint8_t smem[];
-  pdl_wait();   // everything below reads or writes global memory
+  // Launched programmatically, this kernel may start while its predecessor on the stream still runs; nothing the
+  // predecessor may have written is read before pdl_wait().  The shared segment (prompt K/V or register pages), the
+  // block table and cu_seqlens are not among that when the host says so (prefetch_shared): the first tiles of the
+  // key list are then on their way while the predecessor finishes.  The order table IS written just ahead.
+  const bool early_fetch = a.prefetch_shared && a.order == nullptr;
+  if (!early_fetch) {
+    pdl_wait();
+    // (never ahead of the wait: a kernel that lets its successor start only after its own predecessor has ended keeps
+    // every kernel further back ended too, which is what the successor's early fetch relies on)
+    if (a.trigger_early) pdl_launch_dependents();
+  }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // kv heads vary fastest over the grid: the CTAs that read the same rows of the packed K/V tensors (one 256-byte
@@ -82,7 +92,10 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   const int w_lo = row0 / g, w_hi = min((row0 + 15) / g, W - 1);
   const int n_priv = (split == 0) ? (w_hi - w_lo + 1) * step : 0;
   const int n_total = n_shared + n_priv;
-  if (n_total == 0) return;
+  if (n_total == 0) {
+    if (early_fetch) pdl_wait();   // a CTA never ends (which also releases the successor) before the predecessor has
+    return;
+  }
   const int n_tiles = (n_total + KT - 1) / KT;
   const float scale_log2 = a.scale * kLog2e;
 
@@ -133,10 +146,19 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   // tiles in use plus STAGES - 2 in flight.
   constexpr bool PAIR = WALK == STREAM;
   constexpr int PRE = PAIR ? STAGES - 2 : STAGES - 1;   // tiles in flight ahead of the one(s) in use
+  // tiles that lie wholly in the shared segment may be fetched ahead of the wait
+  auto ahead = [&](int s) { return early_fetch && s < n_my && (warp + s * NWARPS + 1) * KT <= n_shared; };
+  if (early_fetch) {
+#pragma unroll
+    for (int s = 0; s < PRE; ++s)
+      if (ahead(s)) issue_tile(warp + s * NWARPS, s);
+    pdl_wait();   // q, k_new, v_new, the private segment and the lineage table are read from here on
+    if (a.trigger_early) pdl_launch_dependents();
+  }
 #pragma unroll
   for (int s = 0; s < PRE; ++s) {
-    if (s < n_my) issue_tile(warp + s * NWARPS, s);
-    cp_async_commit();
+    if (s < n_my && !ahead(s)) issue_tile(warp + s * NWARPS, s);
+    cp_async_commit();   // (the first group also holds every tile fetched ahead of the wait)
   }
 
   // ---- Q fragments, loaded while the first tiles are in flight
@@ -204,7 +226,7 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   // The next kernel on the stream may be scheduled from here on (once every CTA of this grid is past its key
   // loop): releasing it earlier let its CTAs pile up on whichever SMs had room and unbalanced the next launch
   // (55 us against 50 us per prompt-cache layer at the 7B shapes).
-  pdl_launch_dependents();
+  if (!a.trigger_early) pdl_launch_dependents();
   t.reduce_sums();
   __syncthreads();   // all rings are idle: reuse the shared memory
 
@@ -270,6 +292,10 @@ __global__ void __launch_bounds__(NWARPS * 32) decode_mma_kernel(DecodeArgs a) {
   }
 }
 
+#ifndef EARN_DECODE_EARLY_TRIGGER_TILES
+#define EARN_DECODE_EARLY_TRIGGER_TILES 8
+#endif
+
 template <int D, int ST, int NWARPS, Walk WALK>
 cudaError_t launch_d(const DecodeArgs& a, cudaStream_t st) {
   constexpr int smem = Smem<D, ST, NWARPS>::BYTES;
@@ -304,7 +330,20 @@ cudaError_t launch_decode_order(const int32_t* cu_seqlens, int batch, int32_t* o
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-cudaError_t launch_decode_mma(const DecodeArgs& a, int max_shared_len, cudaStream_t st) {
+cudaError_t launch_decode_mma(const DecodeArgs& a0, int max_shared_len, cudaStream_t st) {
+  DecodeArgs a = a0;
+  {
+    // A launch whose CTAs each walk a short list is a chain of latencies (fetch, a few tiles, store), and the next
+    // launch's CTAs fit beside it: let them start at once, so that whatever they may do ahead of their wait (set-up,
+    // the fetch of their shared segment) runs under this launch.  A long list keeps the late trigger: there the CTAs
+    // of the next launch would only take SM resources from this one's streams.
+    const int gq = a.Hq / a.Hkv;
+    const int per_tile = a.beams < (16 + gq - 1) / gq + 1 ? a.beams : (16 + gq - 1) / gq + 1;
+    const int chunk_len = a.plan.n_splits > 1 ? a.plan.chunk : max_shared_len;
+    a.trigger_early = (chunk_len + per_tile * a.step + KT - 1) / KT <= EARN_DECODE_EARLY_TRIGGER_TILES ? 1 : 0;
+  }
+  // A short list under one row tile (the compact cache of a register layer): the whole list at once, see decode_short.cu
+  if (decode_short_supported(a, max_shared_len)) return launch_decode_short(a, max_shared_len, st);
   // Several row tiles (beams x group size > 16): the row tiles of a CTA share one pass over the shared segment.
   if (a.plan.row_tiles > 1) return launch_decode_rows(a, st);
   // One warp per CTA with a deep ring streams best whenever the grid covers the GPU (measured on B200 at the 7B

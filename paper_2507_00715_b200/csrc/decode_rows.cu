@@ -27,7 +27,13 @@ __global__ void __launch_bounds__(RT * 32, MINB) decode_rows_kernel(DecodeArgs a
   constexpr int NT = RT * 32, CH = G::CH, SPW = ST / RT;   // SPW: ring stages a warp owns in phase 2
   static_assert(ST % RT == 0 && SPW >= 1 && NT % CH == 0 && ST >= 4, "ring slices");
   extern __shared__ __align__(128) uint8_t smem[];
-  pdl_wait();   // everything below reads or writes global memory
+  // As in the one-row-tile kernel: with prefetch_shared the first tiles of the shared segment are fetched before the
+  // wait for the kernel ahead on the stream (which cannot have written them); the order table is written just ahead.
+  const bool early_fetch = a.prefetch_shared && a.order == nullptr;
+  if (!early_fetch) {
+    pdl_wait();
+    if (a.trigger_early) pdl_launch_dependents();   // never ahead of the wait (see decode_mma.cu)
+  }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // CTAs are handed out in grid order: with an order table the longest sequences start first and the launch does
@@ -43,7 +49,10 @@ __global__ void __launch_bounds__(RT * 32, MINB) decode_rows_kernel(DecodeArgs a
   const int shared_len = a.src.paged ? a.src.n_regs : (a.cu_seqlens[b + 1] - seq_lo);
   const int key_begin = split * a.plan.chunk;
   const int n_shared = max(min(key_begin + a.plan.chunk, shared_len) - key_begin, 0);
-  if (n_shared == 0 && split != 0) return;   // a split past the end of this sequence
+  if (n_shared == 0 && split != 0) {   // a split past the end of this sequence
+    if (early_fetch) pdl_wait();
+    return;
+  }
   const int n_sh_tiles = (n_shared + KT - 1) / KT;
   const float scale_log2 = a.scale * kLog2e;
 
@@ -74,6 +83,10 @@ __global__ void __launch_bounds__(RT * 32, MINB) decode_rows_kernel(DecodeArgs a
   for (int s = 0; s < ST - 2; ++s) {
     if (s < n_sh_tiles) issue_shared(s, s);
     cp_async_commit();
+  }
+  if (early_fetch) {
+    pdl_wait();   // the lineage table, q, k_new, v_new and the private segment are read from here on
+    if (a.trigger_early) pdl_launch_dependents();
   }
 
   // ---- where the generated tokens of this row tile's beams live: resolved now (lane -> positions lane, lane + 32,
@@ -117,7 +130,7 @@ __global__ void __launch_bounds__(RT * 32, MINB) decode_rows_kernel(DecodeArgs a
     }
   }
   cp_async_wait<0>();
-  pdl_launch_dependents();   // from here on the next kernel on the stream may be scheduled
+  if (!a.trigger_early) pdl_launch_dependents();   // from here on the next kernel on the stream may be scheduled
   __syncthreads();           // the ring is idle: each warp takes its slice
   if (!active) return;
   // ---- Eq. 4: append (split 0).  Nothing in this launch reads the rows it writes (the newest token comes straight

@@ -2,6 +2,7 @@
 #include <cstdio>
 #include <cstring>
 #include <atomic>
+#include <mutex>
 
 #include "earn_common.cuh"
 
@@ -19,6 +20,33 @@ int sm_count() {
   if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) { (void)cudaGetLastError(); return kDefaultSms; }
   if (dev >= 0 && dev < 64) cached[dev].store(n, std::memory_order_relaxed);
   return n;
+}
+
+// ---- what the previous call of this library on a stream launched, remembered per stream (a small table, oldest entry
+// reused).  A decode kernel may fetch its shared segment before the programmatic-launch wait when the kernel ahead of it
+// on the stream (a) cannot have written that segment and (b) itself waited for ITS predecessor before it let its
+// successor start -- true of the decode, register-attention and re-parenting kernels, not of the kernels that write a
+// cache (compaction, the register projection) or of anything this table has not seen.
+enum CallKind { CALL_UNKNOWN = 0, CALL_WRITES_CACHE = 1, CALL_LEAVES_CACHE = 2 };
+static std::mutex g_stream_mutex;
+static struct { earn_stream_t stream; int kind; uint64_t age; bool used; } g_streams[32];
+static uint64_t g_stream_clock = 0;
+
+static void note_call(earn_stream_t stream, int kind) {
+  std::lock_guard<std::mutex> lock(g_stream_mutex);
+  int slot = 0;
+  for (int i = 0; i < 32; ++i) {
+    if (g_streams[i].used && g_streams[i].stream == stream) { slot = i; break; }
+    if (!g_streams[i].used) { slot = i; break; }
+    if (g_streams[i].age < g_streams[slot].age) slot = i;
+  }
+  g_streams[slot].stream = stream; g_streams[slot].kind = kind; g_streams[slot].age = ++g_stream_clock; g_streams[slot].used = true;
+}
+static int last_call(earn_stream_t stream) {
+  std::lock_guard<std::mutex> lock(g_stream_mutex);
+  for (int i = 0; i < 32; ++i)
+    if (g_streams[i].used && g_streams[i].stream == stream) return g_streams[i].kind;
+  return CALL_UNKNOWN;
 }
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -189,6 +217,7 @@ size_t earn_workspace_bytes(const earn_model_t* model, const earn_batch_t* batch
 earn_status_t earn_workspace_init(void* workspace, size_t workspace_bytes, earn_stream_t stream) {
   if (workspace == nullptr || workspace_bytes < (size_t)kStatusBytes || !aligned16(workspace)) return EARN_ERR_WORKSPACE;
   // status word and split tickets start at zero (the partial buffers behind them need no value)
+  note_call(stream, CALL_UNKNOWN);
   return cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
 }
 
@@ -219,6 +248,7 @@ earn_status_t earn_prefill_attn(const earn_model_t* model, const earn_batch_t* b
   a.batch = batch->batch; a.max_seqlen = batch->max_seqlen;
   a.Hq = model->n_q_heads; a.Hkv = model->n_kv_heads; a.D = model->head_dim; a.dtype = model->dtype;
   a.scale = scale_of(model);
+  note_call(stream, CALL_UNKNOWN);
   if (prefill_tc_supported(a, batch->total_tokens)) {
     if (!aligned16(workspace) || workspace_bytes < kStatusBytes + prefill_plan_bytes(*batch)) return EARN_ERR_WORKSPACE;
     return launch_prefill_tc(a, batch->total_tokens,
@@ -252,6 +282,7 @@ earn_status_t earn_compact_kv(const earn_model_t* model, const earn_batch_t* bat
   a.r_head = batch->n_head_reg; a.r_tail = batch->n_tail_reg;
   a.kv_row_bytes = (int)(model->n_kv_heads * model->head_dim * elem_size(model));
   a.q_row_bytes = (int)(model->n_q_heads * model->head_dim * elem_size(model));
+  note_call(stream, CALL_WRITES_CACHE);
   return launch_compact(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
 }
 
@@ -286,6 +317,7 @@ earn_status_t earn_register_qkv(const earn_model_t* model, const earn_batch_t* b
   a.batch = batch->batch; a.R = R; a.r_head = batch->n_head_reg; a.r_tail = batch->n_tail_reg;
   a.Hq = model->n_q_heads; a.Hkv = model->n_kv_heads; a.d_model = proj->d_model;
   a.x_is_compact = proj->x_is_compact != 0; a.max_pos = proj->max_pos; a.rms_eps = proj->rms_eps;
+  note_call(stream, CALL_WRITES_CACHE);
   return launch_register_qkv(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
 }
 
@@ -311,6 +343,7 @@ earn_status_t earn_register_attn(const earn_model_t* model, const earn_batch_t* 
   a.scale = scale_of(model);
   const cudaError_t e = register_mma_supported(a) ? launch_register_mma(a, (cudaStream_t)stream)
                                                   : launch_register_simt(a, (cudaStream_t)stream);
+  note_call(stream, e == cudaSuccess ? CALL_LEAVES_CACHE : CALL_UNKNOWN);
   return e == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
 }
 
@@ -347,6 +380,9 @@ earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* ba
   // Prompt-cache layers of a ragged batch: hand the CTAs out longest sequence first.  The order table (one small
   // launch ahead of the decode kernel) lives in the workspace's prefill-plan area, which holds at least 16 bytes per
   // sequence and is rewritten by every prefill call before it is read.  Worth it when the prompts are long and uneven.
+  // The shared segment may be fetched ahead of the stream-order wait when the call before this one on the stream
+  // launched a kernel that leaves every cache as it found it (see note_call above).
+  a.prefetch_shared = last_call(stream) == CALL_LEAVES_CACHE ? 1 : 0;
   a.order = nullptr;
   if (early && model->dtype == EARN_BF16 && batch->batch >= 2 && batch->batch <= 1024 && batch->max_seqlen >= 1024 &&
       prefill_plan_bytes(*batch) >= sizeof(int32_t) * (size_t)batch->batch) {   // (empty sequences have no plan entry)
@@ -363,6 +399,7 @@ earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* ba
   }
   const cudaError_t e = model->dtype == EARN_BF16 ? launch_decode_mma(a, early ? batch->max_seqlen : batch->n_head_reg + batch->n_tail_reg, (cudaStream_t)stream)
                                                    : launch_decode_simt(a, (cudaStream_t)stream);
+  note_call(stream, e == cudaSuccess ? CALL_LEAVES_CACHE : CALL_UNKNOWN);
   return e == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
 }
 
@@ -371,8 +408,10 @@ earn_status_t earn_beam_reparent(int32_t batch, int32_t beams, int32_t max_new, 
   if (batch < 0 || beams < 1 || max_new < 1 || step < 1 || step > max_new) return EARN_ERR_INVALID_ARG;
   if (batch == 0) return EARN_OK;
   if (parent == nullptr || lineage_out == nullptr || lineage_out == lineage_in_or_null) return EARN_ERR_INVALID_ARG;
-  return launch_beam_reparent(batch, beams, max_new, step, parent, lineage_in_or_null, lineage_out,
-                              (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+  const bool ok = launch_beam_reparent(batch, beams, max_new, step, parent, lineage_in_or_null, lineage_out,
+                                       (cudaStream_t)stream) == cudaSuccess;
+  note_call(stream, ok ? CALL_LEAVES_CACHE : CALL_UNKNOWN);   // an ordinary launch that writes the lineage table only
+  return ok ? EARN_OK : EARN_ERR_CUDA;
 }
 
 }  // extern "C"

@@ -145,10 +145,19 @@ struct DecodeArgs {
   int batch, beams, max_new, step, Hq, Hkv, D, dtype;
   float scale;
   const int32_t* order;        // bf16 kernels: if not null, grid index z is a rank and order[z] the sequence (longest shared segment first)
+  // bf16 kernels: the kernel just ahead of this one on the stream cannot have written the shared segment (nor the block
+  // table, nor cu_seqlens), so its first tiles may be fetched before the programmatic-launch wait
+  int prefetch_shared;
+  // bf16 kernels: let the next kernel on the stream be scheduled as soon as this one starts (short key lists) instead of
+  // after the key loop
+  int trigger_early;
 };
 cudaError_t launch_decode_simt(const DecodeArgs& a, cudaStream_t st);   // fp32 debug path
 // bf16: cp.async ring + mma.sync; max_shared_len = longest shared segment of the batch (picks the ring depth)
 cudaError_t launch_decode_mma(const DecodeArgs& a, int max_shared_len, cudaStream_t st);
+// bf16, one row tile and a list of at most 128 positions (64 at head_dim 64): the whole list in shared memory at once
+bool decode_short_supported(const DecodeArgs& a, int max_shared_len);
+cudaError_t launch_decode_short(const DecodeArgs& a, int max_shared_len, cudaStream_t st);
 // bf16, several row tiles (beams x group size > 16): the row tiles of a CTA share one pass over the shared segment
 cudaError_t launch_decode_rows(const DecodeArgs& a, cudaStream_t st);
 // order[rank] = sequence, by decreasing prompt length (ties by index); batch <= 1024
