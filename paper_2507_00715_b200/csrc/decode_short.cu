@@ -22,6 +22,13 @@ namespace earn {
 namespace {
 using namespace dec;
 
+// Pins a value computed ahead of the stream-order wait: the compiler otherwise sinks pure arithmetic to its first use,
+// which is behind the wait, on the critical path.
+__device__ __forceinline__ void pin(int& x) { asm volatile("" : "+r"(x)); }
+__device__ __forceinline__ void pin(int64_t& x) { asm volatile("" : "+l"(x)); }
+template <typename T>
+__device__ __forceinline__ void pin(T*& x) { asm volatile("" : "+l"(x)); }
+
 template <int D, int NW>
 struct ShortSmem {
   using G = Geo<D>;
@@ -62,30 +69,105 @@ __global__ void __launch_bounds__(NW * 32) decode_short_kernel(DecodeArgs a) {
   const bf16* kg = reinterpret_cast<const bf16*>(a.src.k);
   const bf16* vg = reinterpret_cast<const bf16*>(a.src.v);
 
-  // ---- copies: thread -> (list position r_t + i * RPP, 16-byte chunk c_t), K and V alike; position p sits in row
-  // p % 16 of tile p / 16
-  const int c_t = threadIdx.x % CH, r_t = threadIdx.x / CH;
+  // ---- where every row lives, worked out ONCE per row (thread p for list position p, the next 16 threads for the
+  // query rows) and passed through a table in shared memory: the divisions and 64-bit products of this arithmetic,
+  // done by every thread for each of its pieces, were 2 us of a CTA's life.  The table sits in the score area, which
+  // nothing else uses before the first barrier behind the wait.
   const bool affine = !a.src.paged || a.src.block_table == nullptr;
   const int64_t row_base = a.src.paged ? (int64_t)b * a.src.pages_per_seq * EARN_PAGE_TOKENS : (int64_t)seq_lo;
+  int64_t* tab_off = reinterpret_cast<int64_t*>(sc);          // [NW*16] element offset of the row (this kv head) in its tensor
+  int64_t* tab_q = tab_off + NW * 16;                          // [16] element offset of the query / output row, -1: none
+  int* tab_key = reinterpret_cast<int*>(tab_q + 16);           // [NW*16] -1: shared or zero row; -3: newest token; else j * max_new + t
+  int* tab_beam = tab_key + NW * 16;                           // [16] beam of the query row
+  static_assert((NW * 16 + 16) * 12 <= S::SC_B, "table fits the score area");
+  if ((int)threadIdx.x < NW * 16) {
+    const int p = threadIdx.x;
+    int64_t off = 0;
+    int key = -1;
+    if (p < n_shared) {
+      off = ((affine ? row_base + p : key_row(a.src, b, p)) * a.Hkv + kvh) * D;
+    } else if (p < n_total) {
+      const int pk = p - n_shared, w = pk / step, t = pk - w * step;
+      const int64_t j = (int64_t)b * W + w;
+      if (t == step - 1) {
+        key = -3;
+        off = (j * a.Hkv + kvh) * D;
+      } else {
+        key = (int)(j * a.max_new + t);
+        off = ((j * a.max_new + t) * a.Hkv + kvh) * D;   // identity lineage; corrected behind the wait otherwise
+      }
+    }
+    tab_off[p] = off;
+    tab_key[p] = key;
+  } else if ((int)threadIdx.x < NW * 16 + 16) {
+    const int r = threadIdx.x - NW * 16;
+    tab_q[r] = rm.offset(r, D);
+    tab_beam[r] = r / g;
+  }
+  __syncthreads();
+
+  // ---- copies: thread -> (list position r_t + i * RPP, 16-byte chunk c_t), K and V alike; position p sits in row
+  // p % 16 of tile p / 16.  Shared rows are fetched now; rows past the list, and query rows past W*g, are zeroed with
+  // plain stores; the rest waits.
+  const int c_t = threadIdx.x % CH, r_t = threadIdx.x / CH;
   auto dst_of = [&](int p) { return kv + (uint32_t)(p >> 4) * G::STAGE_B + (uint32_t)(p & 15) * G::PITCH + (uint32_t)c_t * 16; };
+  int64_t p_off[PASSES];
+  int p_key[PASSES];
 #pragma unroll
   for (int i = 0; i < PASSES; ++i) {
     const int p = r_t + i * RPP;
+    p_off[i] = tab_off[p] + c_t * 8;
+    p_key[i] = tab_key[p];
     if (p < n_shared) {
-      const int64_t row = affine ? row_base + p : key_row(a.src, b, p);
-      const int64_t off = (row * a.Hkv + kvh) * D + c_t * 8;
-      cp_async16(dst_of(p), kg + off);
-      cp_async16(dst_of(p) + G::TILE_B, vg + off);
+      cp_async16(dst_of(p), kg + p_off[i]);
+      cp_async16(dst_of(p) + G::TILE_B, vg + p_off[i]);
+    } else if (p >= n_total) {
+      uint8_t* z = smem + (p >> 4) * G::STAGE_B + (p & 15) * G::PITCH + c_t * 16;
+      *reinterpret_cast<uint4*>(z) = make_uint4(0u, 0u, 0u, 0u);
+      *reinterpret_cast<uint4*>(z + G::TILE_B) = make_uint4(0u, 0u, 0u, 0u);
     }
   }
-  // where this thread's query pieces, and the lane's two output rows, live
   int64_t q_off[QPASSES];
 #pragma unroll
-  for (int i = 0; i < QPASSES; ++i) q_off[i] = rm.offset(r_t + i * RPP, D);
+  for (int i = 0; i < QPASSES; ++i) {
+    q_off[i] = tab_q[r_t + i * RPP];
+    if (q_off[i] < 0)
+      *reinterpret_cast<uint4*>(smem + S::KV_B + (r_t + i * RPP) * G::PITCH + c_t * 16) = make_uint4(0u, 0u, 0u, 0u);
+  }
   const int r0 = lane >> 2, r1 = r0 + 8, c2 = (lane & 3) * 2;
-  const int64_t o_off0 = rm.offset(r0, D), o_off1 = rm.offset(r1, D);
-  // generated tokens a row may see: its own beam's, at list positions vis .. vis + step - 1
-  const int vis0 = n_shared + (r0 / g) * step, vis1 = n_shared + (r1 / g) * step;
+  int64_t o_off0 = tab_q[r0], o_off1 = tab_q[r1];
+  int seen_bits = 0;   // bit n * 4 + e: element e of 8-column block n of this warp's score tile is visible to its row
+  {
+    // generated tokens a row may see: its own beam's, at list positions vis .. vis + step - 1
+    const int vis0 = n_shared + tab_beam[r0] * step, vis1 = n_shared + tab_beam[r1] * step;
+#pragma unroll
+    for (int n = 0; n < 2; ++n)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int p = warp * KT + n * 8 + c2 + (e & 1), v0 = e >= 2 ? vis1 : vis0;
+        if (p < n_shared || (p >= v0 && p < v0 + step)) seen_bits |= 1 << (n * 4 + e);
+      }
+  }
+  // Eq. 4, append: the newest token of beam w sits at list position n_shared + w * step + step - 1; piece i of the
+  // W * 2 * CH 16-byte pieces goes from the tile in shared memory to the private segment.  The first piece of each
+  // thread (all of them up to four beams) is addressed here, ahead of the wait.
+  auto app_piece = [&](int i, const uint8_t*& src, bf16*& dst) {
+    const int w = i / (2 * CH), c = i % (2 * CH), p = n_shared + w * step + step - 1;
+    src = smem + (p >> 4) * G::STAGE_B + (c >= CH ? G::TILE_B : 0) + (p & 15) * G::PITCH + (c % CH) * 16;
+    dst = reinterpret_cast<bf16*>(c >= CH ? a.v_priv : a.k_priv) +
+          ((((int64_t)b * W + w) * a.max_new + (step - 1)) * a.Hkv + kvh) * D + (c % CH) * 8;
+  };
+  const uint8_t* app_src = nullptr;
+  bf16* app_dst = nullptr;
+  if ((int)threadIdx.x < W * 2 * CH) app_piece(threadIdx.x, app_src, app_dst);
+  {
+    pin(app_src); pin(app_dst);
+    pin(o_off0); pin(o_off1); pin(seen_bits);
+#pragma unroll
+    for (int i = 0; i < PASSES; ++i) { pin(p_off[i]); pin(p_key[i]); }
+#pragma unroll
+    for (int i = 0; i < QPASSES; ++i) pin(q_off[i]);
+  }
 
   if (early_fetch) {
     pdl_wait();   // q, k_new, v_new, the private segment and the lineage table are read from here on
@@ -94,38 +176,37 @@ __global__ void __launch_bounds__(NW * 32) decode_short_kernel(DecodeArgs a) {
   {
     const bf16* qg = reinterpret_cast<const bf16*>(a.q);
 #pragma unroll
-    for (int i = 0; i < QPASSES; ++i)   // rows past W*g become zero
-      cp_async16(qs + (uint32_t)(r_t + i * RPP) * G::PITCH + (uint32_t)c_t * 16, qg + (q_off[i] < 0 ? 0 : q_off[i]) + c_t * 8,
-                 q_off[i] < 0 ? 0 : 16);
-    const bf16* kp[3] = {kg, reinterpret_cast<const bf16*>(a.k_priv), reinterpret_cast<const bf16*>(a.k_new)};
-    const bf16* vp[3] = {vg, reinterpret_cast<const bf16*>(a.v_priv), reinterpret_cast<const bf16*>(a.v_new)};
+    for (int i = 0; i < QPASSES; ++i)   // (a pass without query rows is skipped by every thread alike)
+      if (i * RPP < rm.n_rows && q_off[i] >= 0)
+        cp_async16(qs + (uint32_t)(r_t + i * RPP) * G::PITCH + (uint32_t)c_t * 16, qg + q_off[i] + c_t * 8);
+    const bf16 *kpriv = reinterpret_cast<const bf16*>(a.k_priv), *vpriv = reinterpret_cast<const bf16*>(a.v_priv);
+    const bf16 *knew = reinterpret_cast<const bf16*>(a.k_new), *vnew = reinterpret_cast<const bf16*>(a.v_new);
 #pragma unroll
     for (int i = 0; i < PASSES; ++i) {
+      // a pass that holds no generated token is skipped by every thread alike: a compare and a branch, no more
+      if ((i + 1) * RPP <= n_shared || i * RPP >= n_total) continue;
       const int p = r_t + i * RPP;
-      if (p >= n_shared) {
-        int which = 1;
-        const bool ok = p < n_total;
-        const int64_t off = ok ? private_row<D>(a, b, kvh, 0, p - n_shared, which) + c_t * 8 : 0;
-        cp_async16(dst_of(p), (which == 2 ? kp[2] : kp[1]) + off, ok ? 16 : 0);   // past the list: zero rows
-        cp_async16(dst_of(p) + G::TILE_B, (which == 2 ? vp[2] : vp[1]) + off, ok ? 16 : 0);
+      if (p_key[i] == -1) continue;
+      int64_t off = p_off[i];
+      if (a.lineage != nullptr && p_key[i] >= 0) {   // the token lives in the slab of the beam that generated it
+        const int t = p_key[i] % a.max_new;
+        const int64_t slab = min(max(a.lineage[p_key[i]], 0), a.batch * W - 1);
+        off = ((slab * a.max_new + t) * a.Hkv + kvh) * D + c_t * 8;
       }
+      const bool fresh = p_key[i] == -3;
+      cp_async16(dst_of(p), (fresh ? knew : kpriv) + off);
+      cp_async16(dst_of(p) + G::TILE_B, (fresh ? vnew : vpriv) + off);
     }
   }
   cp_async_commit();
   cp_async_wait<0>();
   __syncthreads();
 
-  // ---- Eq. 4, append: the newest token of beam w sits at list position n_shared + w * step + step - 1
-  {
-    bf16* kpriv = reinterpret_cast<bf16*>(a.k_priv);
-    bf16* vpriv = reinterpret_cast<bf16*>(a.v_priv);
-    for (int i = threadIdx.x; i < W * 2 * CH; i += NT) {
-      const int w = i / (2 * CH), c = i % (2 * CH), p = n_shared + w * step + step - 1;
-      const uint8_t* srcp = smem + (p >> 4) * G::STAGE_B + (c >= CH ? G::TILE_B : 0) + (p & 15) * G::PITCH + (c % CH) * 16;
-      const int64_t j = (int64_t)b * W + w;
-      *reinterpret_cast<uint4*>((c >= CH ? vpriv : kpriv) + ((j * a.max_new + (step - 1)) * a.Hkv + kvh) * D + (c % CH) * 8) =
-          *reinterpret_cast<const uint4*>(srcp);
-    }
+  // ---- Eq. 4, append, from the tile in shared memory
+  if (app_src != nullptr) *reinterpret_cast<uint4*>(app_dst) = *reinterpret_cast<const uint4*>(app_src);
+  for (int i = threadIdx.x + NT; i < W * 2 * CH; i += NT) {
+    app_piece(i, app_src, app_dst);
+    *reinterpret_cast<uint4*>(app_dst) = *reinterpret_cast<const uint4*>(app_src);
   }
 
   // ---- S = Q K^T for tile `warp`; scaled scores (log2 domain) into shared memory, invisible positions as -inf
@@ -150,11 +231,7 @@ __global__ void __launch_bounds__(NW * 32) decode_short_kernel(DecodeArgs a) {
     for (int n = 0; n < 2; ++n) {
       float x[4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int p = warp * KT + n * 8 + c2 + (e & 1), v0 = e >= 2 ? vis1 : vis0;
-        const bool seen = p < n_shared || (p >= v0 && p < v0 + step);
-        x[e] = seen ? (s[n][e] + s2[n][e]) * scale_log2 : -INFINITY;
-      }
+      for (int e = 0; e < 4; ++e) x[e] = (seen_bits >> (n * 4 + e)) & 1 ? (s[n][e] + s2[n][e]) * scale_log2 : -INFINITY;
       *reinterpret_cast<float2*>(sc + r0 * S::SC_PITCH + warp * KT + n * 8 + c2) = make_float2(x[0], x[1]);
       *reinterpret_cast<float2*>(sc + r1 * S::SC_PITCH + warp * KT + n * 8 + c2) = make_float2(x[2], x[3]);
     }
