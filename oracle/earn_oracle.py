@@ -26,6 +26,8 @@ What pins each function (see tests/test_oracle_pins.py):
                           "project every row then gather" = "gather then project" (Eq. 2 acts per token)
   rope_tables           : closed-form angles (D = 8, theta = 10000: 1, 0.1, 0.01, 0.001 rad per position)
   attention_scores, sparsity, sinks : the scalar definitions of Eq. 14-15 by hand
+  beam_topk             : python's sorted() on (score, index) tuples; hand-made cases (a dominant beam, exact ties,
+                          the first step with one live beam); greedy decoding (one beam) = argmax
 Attention values have no printed worked example in the paper, so beyond those
 pins they are parity unpinned.
 """
@@ -309,6 +311,40 @@ class DecodeState:
     def entries(self, b: int) -> int:
         """KV entries one beam of sequence b reads in this layer (per kv head)."""
         return self.shared_k[b].shape[0] + len(self.priv_k[b * self.beams])
+
+
+# --------------------------------------------------------------------------
+# Appendix A.3: item identifiers are generated by beam search (beam size 20).  The paper gives the beam size only; the
+# selection rule is that of ordinary beam search: after a step the W continuations (beam, token) with the highest
+# cumulative log-probability survive.
+# --------------------------------------------------------------------------
+def beam_topk(logprobs, beam_scores, beams: int, n_live: Optional[int] = None):
+    """logprobs [B*W, V] (log-probability of every token after every beam), beam_scores [B*W] (cumulative
+    log-probability of every beam so far) -> (parent int32 [B*W], token int32 [B*W], score float32 [B*W]).
+
+    Candidate (w, v) of a sequence scores beam_scores[w] + logprobs[w, v], the sum taken in float32 (the precision
+    the selection is made in; the inputs are float32).  Only beams w < n_live of every sequence offer candidates
+    (at the first step all beams hold the same history, so n_live = 1); default: all.  Output slot i of a sequence gets
+    the i-th best candidate: higher score first, equal scores in increasing order of the flat candidate index
+    w * V + v.  parent is the beam index within the sequence.
+    """
+    lp = np.asarray(logprobs, dtype=np.float32)
+    sc = np.asarray(beam_scores, dtype=np.float32)
+    n, vocab = lp.shape
+    live = beams if n_live is None else int(n_live)
+    if not (1 <= live <= beams) or live * vocab < beams:
+        raise ValueError("need at least `beams` candidates per sequence")
+    parent = np.zeros(n, dtype=np.int32)
+    token = np.zeros(n, dtype=np.int32)
+    score = np.zeros(n, dtype=np.float32)
+    for b in range(n // beams):
+        rows = slice(b * beams, b * beams + live)
+        cand = (sc[rows, None] + lp[rows]).astype(np.float32).reshape(-1)       # flat index w * V + v
+        order = np.argsort(-cand, kind="stable")[:beams]                          # stable: ties keep index order
+        parent[b * beams:(b + 1) * beams] = order // vocab
+        token[b * beams:(b + 1) * beams] = order % vocab
+        score[b * beams:(b + 1) * beams] = cand[order]
+    return parent, token, score
 
 
 # --------------------------------------------------------------------------

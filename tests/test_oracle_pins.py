@@ -446,3 +446,42 @@ def test_attention_scores_by_hand():
     z = math.fsum(math.exp(s) for s in logits)
     np.testing.assert_allclose(p, [math.exp(s) / z for s in logits], atol=1e-15)
     assert abs(p.sum() - 1.0) < 1e-15
+
+
+# ---------------------------------------------------------------- beam selection (Appendix A.3: beam search)
+def test_beam_topk_matches_sorted_tuples_and_hand_cases():
+    rng = np.random.default_rng(13)
+    B, W, V = 3, 4, 11
+    lp = rng.standard_normal((B * W, V)).astype(np.float32)
+    lp[2, 5] = lp[1, 3] = lp[0, 7]                      # plant exact ties inside sequence 0 (equal beam scores below)
+    sc = rng.standard_normal(B * W).astype(np.float32)
+    sc[0] = sc[1] = sc[2]
+    parent, token, score = orc.beam_topk(lp, sc, W)
+    for b in range(B):
+        cands = []
+        for w in range(W):
+            for v in range(V):
+                cands.append((-float(np.float32(sc[b * W + w]) + np.float32(lp[b * W + w, v])), w * V + v))
+        best = sorted(cands)[:W]                        # higher score first, then lower flat index
+        assert [c[1] // V for c in best] == list(parent[b * W:(b + 1) * W])
+        assert [c[1] % V for c in best] == list(token[b * W:(b + 1) * W])
+        assert [np.float32(-c[0]) for c in best] == list(score[b * W:(b + 1) * W])
+    # one beam far ahead of the others: every survivor continues it, tokens in order of their log-probability
+    sc2 = np.array([0.0, 100.0, 0.0, 0.0], dtype=np.float32)
+    lp2 = rng.standard_normal((4, 9)).astype(np.float32)
+    p2, t2, s2 = orc.beam_topk(lp2, sc2, 4)
+    assert list(p2) == [1, 1, 1, 1] and list(t2) == list(np.argsort(-lp2[1], kind="stable")[:4])
+    # all candidates equal: the first W flat indices, in order
+    p3, t3, s3 = orc.beam_topk(np.zeros((3, 5), np.float32), np.zeros(3, np.float32), 3)
+    assert list(p3) == [0, 0, 0] and list(t3) == [0, 1, 2] and not s3.any()
+    # first step: only beam 0 is live, whatever the other rows hold
+    lp4 = rng.standard_normal((4, 9)).astype(np.float32)
+    lp4[1:] += 50.0
+    p4, t4, _ = orc.beam_topk(lp4, np.zeros(4, np.float32), 4, n_live=1)
+    assert list(p4) == [0, 0, 0, 0] and list(t4) == list(np.argsort(-lp4[0], kind="stable")[:4])
+    # one beam: greedy decoding, the arg max
+    lp5 = rng.standard_normal((6, 13)).astype(np.float32)
+    p5, t5, s5 = orc.beam_topk(lp5, np.zeros(6, np.float32), 1)
+    assert not p5.any() and list(t5) == list(lp5.argmax(axis=1)) and np.array_equal(s5, lp5.max(axis=1))
+    with pytest.raises(ValueError):
+        orc.beam_topk(np.zeros((4, 3), np.float32), np.zeros(4, np.float32), 4, n_live=1)   # 3 candidates for 4 slots
