@@ -26,6 +26,7 @@ sys.path.insert(0, ROOT)
 from paper_2507_00715_b200 import replicas, workloads as wl  # noqa: E402
 
 METRIC = "EARN attn tokens/s/GPU (prefill+decode, 7B GQA)"
+BEAM_VOCAB = 32000   # vocabulary the beam-selection kernel is timed on (the size of the paper's multi-head backbone's)
 UNIT = "tokens/s"
 
 
@@ -122,6 +123,7 @@ def algorithmic(w: wl.Workload):
     qo = 2 * B * W * Hq * D * es + 4 * B * W * Hkv * D * es
     out["decode_compact"] = dict(flops=4.0 * D * Hq * B * W * (R + s), bytes=float(2 * B * (R + W * s) * Hkv * D * es + qo))
     out["decode_full"] = dict(flops=4.0 * D * Hq * W * (tot + B * s), bytes=float(2 * (tot + B * W * s) * Hkv * D * es + qo))
+    out["beam_topk"] = dict(flops=0.0, bytes=float(B * W * BEAM_VOCAB * 4 + B * W * 16))
     return out
 
 
@@ -322,6 +324,17 @@ class GpuJob:
                                                                               ses.x_norm, caches[l], self.q_reg, ses.workspace)
                                                      for i, l in enumerate(late)], len(late))
                 del x, wts
+        if w.beams > 1:
+            # beam selection between decode steps (not part of the timed step, which has no output layer to produce
+            # log-probabilities): every log-probability read once, B * W * V * 4 bytes
+            vocab = BEAM_VOCAB
+            lp = wl.beam_logprobs(w, 1, vocab, self.dev)
+            rows = w.batch * w.beams
+            sc = [torch.zeros(rows, device=self.dev), torch.zeros(rows, device=self.dev)]
+            par, tok = (torch.zeros(rows, dtype=torch.int32, device=self.dev) for _ in range(2))
+            ws = torch.empty(self.B.earn_beam_topk_workspace_bytes(w.batch, w.beams, vocab), dtype=torch.uint8, device=self.dev)
+            res["beam_topk"] = timed(lambda: self.B.earn_beam_topk(w.batch, w.beams, w.beams, vocab, lp, sc[0], par, tok, sc[1], ws), 1)
+            del lp, ws
         if w.decode_steps > 0:
             s = w.decode_steps
             if late:

@@ -214,6 +214,24 @@ earn_status_t earn_beam_reparent(int32_t batch, int32_t beams, int32_t max_new, 
                                  const int32_t* parent, const int32_t* lineage_in_or_null,
                                  int32_t* lineage_out, earn_stream_t stream);
 
+/* Beam selection between decode steps (Appendix A.3: identifiers are generated by beam search, beam size 20; the paper
+ * gives the beam size only, the rule is that of ordinary beam search).  For every sequence, of the n_live * vocab
+ * continuations (beam w < n_live, token v), scored beam_scores[b*W + w] + logprobs[b*W + w][v] in fp32, the W best
+ * survive: higher score first, equal scores by increasing flat index w * vocab + v.  Slot i of the sequence receives the
+ * i-th best: parent[b*W + i] = w (ready for earn_beam_reparent), token[b*W + i] = v, new_scores[b*W + i] = its score.
+ * n_live = 1 at the first step (all beams hold the same history), W afterwards.  A decode step is then
+ * earn_beam_topk -> earn_beam_reparent -> earn_decode_attn per layer, with no host round trip.
+ * logprobs: device fp32 [B*W, vocab], no NaN (-inf marks a forbidden token); beam_scores: device fp32 [B*W] or NULL
+ * (zeros); parent, token: device int32 [B*W]; new_scores: device fp32 [B*W], must not alias beam_scores.
+ * workspace: device, at least earn_beam_topk_workspace_bytes(batch, beams, vocab) bytes, 16-byte aligned; no need to
+ * initialise it.  Errors: beams outside [1, 32], n_live outside [1, beams], n_live * vocab < beams -> INVALID_ARG;
+ * beams * vocab beyond 2^31 - 1 or beyond what the two selection levels hold (3.3 M candidates at 20 beams)
+ * -> UNSUPPORTED; workspace NULL / too small -> WORKSPACE. */
+size_t earn_beam_topk_workspace_bytes(int32_t batch, int32_t beams, int32_t vocab);
+earn_status_t earn_beam_topk(int32_t batch, int32_t beams, int32_t n_live, int32_t vocab, const float* logprobs,
+                             const float* beam_scores_or_null, int32_t* parent, int32_t* token, float* new_scores,
+                             void* workspace, size_t workspace_bytes, earn_stream_t stream);
+
 /* Number of kernels this library has launched in this process so far (host counter, all streams). */
 uint64_t earn_launch_count(void);
 

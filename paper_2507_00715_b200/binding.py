@@ -69,6 +69,9 @@ SYMBOLS = {
                                           C.c_void_p]),
     "earn_beam_reparent": (C.c_int, [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.c_void_p]),
+    "earn_beam_topk_workspace_bytes": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int32]),
+    "earn_beam_topk": (C.c_int, [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                 C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "earn_launch_count": (C.c_uint64, []),
     "earn_status_string": (C.c_char_p, [C.c_int]),
     "earn_version": (C.c_int32, []),
@@ -236,3 +239,15 @@ def earn_decode_attn_static(model, batch: Batch, layer, step, q, k_new, v_new, c
 def earn_beam_reparent(batch: int, beams: int, max_new: int, step: int, parent, lineage_in, lineage_out) -> None:
     _check(lib().earn_beam_reparent(batch, beams, max_new, step, _ptr(parent), _ptr(lineage_in), _ptr(lineage_out),
                                     _stream()), "earn_beam_reparent")
+
+
+def earn_beam_topk_workspace_bytes(batch: int, beams: int, vocab: int) -> int:
+    return lib().earn_beam_topk_workspace_bytes(batch, beams, vocab)
+
+
+def earn_beam_topk(batch: int, beams: int, n_live: int, vocab: int, logprobs, beam_scores, parent, token, new_scores,
+                   workspace) -> None:
+    """logprobs fp32 [B*W, vocab], beam_scores fp32 [B*W] or None -> parent, token int32 [B*W], new_scores fp32 [B*W]."""
+    p, n = _ws(workspace)
+    _check(lib().earn_beam_topk(batch, beams, n_live, vocab, _ptr(logprobs), _ptr(beam_scores), _ptr(parent), _ptr(token),
+                                _ptr(new_scores), p, n, _stream()), "earn_beam_topk")

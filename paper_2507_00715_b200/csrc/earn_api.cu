@@ -414,4 +414,28 @@ earn_status_t earn_beam_reparent(int32_t batch, int32_t beams, int32_t max_new, 
   return ok ? EARN_OK : EARN_ERR_CUDA;
 }
 
+size_t earn_beam_topk_workspace_bytes(int32_t batch, int32_t beams, int32_t vocab) {
+  if (batch < 0 || beams < 1 || beams > 32 || vocab < 1 || !beam_topk_supported(beams, vocab)) return 256;
+  return beam_topk_workspace(batch, beams, vocab);
+}
+
+earn_status_t earn_beam_topk(int32_t batch, int32_t beams, int32_t n_live, int32_t vocab, const float* logprobs,
+                             const float* beam_scores_or_null, int32_t* parent, int32_t* token, float* new_scores,
+                             void* workspace, size_t workspace_bytes, earn_stream_t stream) {
+  if (batch < 0 || beams < 1 || beams > 32 || vocab < 1 || n_live < 1 || n_live > beams) return EARN_ERR_INVALID_ARG;
+  if ((int64_t)n_live * vocab < beams) return EARN_ERR_INVALID_ARG;   // fewer continuations than beams to fill
+  if (batch > 65535 || !beam_topk_supported(beams, vocab)) return EARN_ERR_UNSUPPORTED;
+  if (batch == 0) return EARN_OK;
+  if (!logprobs || !parent || !token || !new_scores || new_scores == beam_scores_or_null) return EARN_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(logprobs) | reinterpret_cast<uintptr_t>(parent) | reinterpret_cast<uintptr_t>(token) |
+       reinterpret_cast<uintptr_t>(new_scores) | reinterpret_cast<uintptr_t>(beam_scores_or_null)) & 3u)
+    return EARN_ERR_INVALID_ARG;
+  if (workspace == nullptr || !aligned16(workspace) || workspace_bytes < beam_topk_workspace(batch, beams, vocab))
+    return EARN_ERR_WORKSPACE;
+  const bool ok = launch_beam_topk(batch, beams, n_live, vocab, logprobs, beam_scores_or_null, parent, token, new_scores,
+                                   workspace, (cudaStream_t)stream) == cudaSuccess;
+  note_call(stream, ok ? CALL_LEAVES_CACHE : CALL_UNKNOWN);   // ordinary launches that write the beam tables only
+  return ok ? EARN_OK : EARN_ERR_CUDA;
+}
+
 }  // extern "C"

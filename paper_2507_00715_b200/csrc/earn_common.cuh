@@ -190,6 +190,12 @@ cudaError_t launch_register_qkv(const RegisterQkvArgs& a, cudaStream_t st);
 cudaError_t launch_beam_reparent(int batch, int beams, int max_new, int step, const int32_t* parent,
                                  const int32_t* lineage_in, int32_t* lineage_out, cudaStream_t st);
 
+// beam selection (top W of n_live * vocab continuations per sequence)
+bool beam_topk_supported(int beams, int vocab);
+size_t beam_topk_workspace(int batch, int beams, int vocab);
+cudaError_t launch_beam_topk(int batch, int beams, int n_live, int vocab, const float* logprobs, const float* beam_scores,
+                             int32_t* parent, int32_t* token, float* new_scores, void* workspace, cudaStream_t st);
+
 // ---- element helpers ----
 template <typename T> struct Elem;
 template <> struct Elem<float> {

@@ -101,7 +101,8 @@ CONFIGS["paper_gqa"] = Workload("paper_gqa", batch=48, n_layers=28, split_k=7, n
                                 beams=20, seed=7)
 LONG_SPLIT_SWEEP = (2, 4, 8, 16)
 
-_TAG = {"q": 1, "k": 2, "v": 3, "dq": 4, "dk": 5, "dv": 6, "len": 7, "u": 8, "parent": 9, "x": 10, "wn": 11, "wqkv": 12}
+_TAG = {"q": 1, "k": 2, "v": 3, "dq": 4, "dk": 5, "dv": 6, "len": 7, "u": 8, "parent": 9, "x": 10, "wn": 11, "wqkv": 12,
+        "logits": 13}
 
 
 def _seed_for(w: Workload, tag: str, layer: int = 0, step: int = 0) -> int:
@@ -197,3 +198,19 @@ def beam_parents(w: Workload, step: int) -> np.ndarray:
         return np.tile(np.arange(w.beams, dtype=np.int32), w.batch)
     rng = np.random.Generator(np.random.Philox(_seed_for(w, "parent", 0, step)))
     return rng.integers(0, w.beams, size=w.batch * w.beams).astype(np.int32)
+
+
+def beam_logprobs(w: Workload, step: int, vocab: int, device="cpu", allowed: int = 0) -> torch.Tensor:
+    """Token log-probabilities after every beam at a decode step, fp32 [B*W, vocab]: the log-softmax of logits
+    ~ 3 N(0,1) (there is no model here to produce them).  With allowed > 0 only `allowed` tokens per row, drawn from the
+    seed, keep a finite value (identifier generation restricted to valid tokens); the rest are -inf."""
+    rows = w.batch * w.beams
+    logits = 3.0 * _randn((rows, vocab), _seed_for(w, "logits", 0, step), device)
+    if allowed > 0:
+        g = torch.Generator()
+        g.manual_seed(_seed_for(w, "logits", 1, step))
+        keep = torch.zeros(rows, vocab, dtype=torch.bool)
+        for r in range(rows):
+            keep[r, torch.randperm(vocab, generator=g)[:allowed]] = True
+        logits = torch.where(keep.to(device), logits, torch.full_like(logits, float("-inf")))
+    return torch.log_softmax(logits, dim=-1)

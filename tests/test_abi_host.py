@@ -133,6 +133,29 @@ def test_host_validation_decode_static(lib):
     assert lib.earn_launch_count() == n0
 
 
+def test_host_validation_beam_topk(lib):
+    def call(batch=2, beams=4, n_live=4, vocab=100, lp=0x1000, scores=0x2000, new=0x3000, ws=0x4000, ws_bytes=1 << 20):
+        return lib.earn_beam_topk(batch, beams, n_live, vocab, lp, scores, 0x5000, 0x6000, new, ws, ws_bytes, None)
+
+    n0 = lib.earn_launch_count()
+    assert call(beams=0) == B.EARN_ERR_INVALID_ARG
+    assert call(beams=33) == B.EARN_ERR_INVALID_ARG
+    assert call(n_live=0) == B.EARN_ERR_INVALID_ARG
+    assert call(n_live=5) == B.EARN_ERR_INVALID_ARG
+    assert call(beams=4, n_live=1, vocab=3) == B.EARN_ERR_INVALID_ARG      # three continuations cannot fill four beams
+    assert call(lp=0) == B.EARN_ERR_INVALID_ARG
+    assert call(lp=0x1002) == B.EARN_ERR_INVALID_ARG                        # fp32 pointers are 4-byte aligned
+    assert call(new=0x2000) == B.EARN_ERR_INVALID_ARG                       # the new scores would overwrite the old in place
+    assert call(ws=0) == B.EARN_ERR_WORKSPACE
+    assert call(beams=20, n_live=20, vocab=152064, ws_bytes=256) == B.EARN_ERR_WORKSPACE
+    assert call(beams=32, n_live=32, vocab=1 << 20) == B.EARN_ERR_UNSUPPORTED   # more chunks than the second level holds
+    assert call(batch=0) == B.EARN_OK
+    assert lib.earn_launch_count() == n0
+    # one chunk needs no partial lists; 20 beams x 152064 tokens = 372 chunks of 8192 candidates, 20 (score, index) pairs each
+    assert lib.earn_beam_topk_workspace_bytes(48, 20, 100) == 256
+    assert lib.earn_beam_topk_workspace_bytes(48, 20, 152064) >= 48 * 372 * 20 * 8
+
+
 def test_host_validation_register_qkv(lib):
     m = B.make_model(4, 2, 8, 2, 128, "bf16")
     b = FakeBatch([40, 50], 10, 10)
