@@ -83,13 +83,21 @@ typedef struct {
   const int32_t* block_table; /* device [B, pages_per_seq] page numbers, or NULL: page p of sequence b is b*pages_per_seq+p */
   int32_t pages_per_seq;      /* >= ceil(R / 16) */
   int32_t n_pages;            /* pages allocated in k_shared / v_shared (bounds the block table) */
-  void* k_priv;               /* device [B*beams, max_new, Hkv, D] generated keys; row (j, t) is written at step t+1 by beam j */
+  void* k_priv;               /* device [B*beams, max_new, Hkv, D] generated keys; row (j, t) is written at step t+1 by beam j
+                                 (with priv_block_table: device [n_priv_pages, 16, Hkv, D], see below) */
   void* v_priv;               /* device, same shape */
   const int32_t* lineage;     /* device [B*beams, max_new] or NULL (identity): lineage[j][t] = slab holding token t of the
                                  history of beam j, maintained by earn_beam_reparent */
   int32_t beams;              /* W >= 1 */
   int32_t max_new;            /* T: capacity of the private segment in tokens */
   int32_t* reg_idx;           /* device [B, R] or NULL: earn_compact_kv writes the gathered source positions here */
+  /* Optional page table of the private segment (NULL: the flat slabs above).  With a table, token t generated by beam j
+   * lives in slot t % 16 of page priv_block_table[j * priv_pages_per_beam + t / 16] of k_priv / v_priv, so a beam costs
+   * pages as it grows (one per 16 generated tokens) instead of a max_new-row slab up front.  The caller allocates a
+   * beam's next page before the decode step that writes into it. */
+  const int32_t* priv_block_table; /* device [B*beams, priv_pages_per_beam] or NULL */
+  int32_t priv_pages_per_beam;     /* >= ceil(max_new / 16) */
+  int32_t n_priv_pages;            /* pages allocated in k_priv / v_priv (bounds the table) */
 } earn_cache_t;
 
 /* Bytes of caller-provided scratch that cover every call below for this model, batch and beam

@@ -39,7 +39,8 @@ class EarnCache(C.Structure):
     _fields_ = [("k_shared", C.c_void_p), ("v_shared", C.c_void_p), ("block_table", C.c_void_p),
                 ("pages_per_seq", C.c_int32), ("n_pages", C.c_int32),
                 ("k_priv", C.c_void_p), ("v_priv", C.c_void_p), ("lineage", C.c_void_p),
-                ("beams", C.c_int32), ("max_new", C.c_int32), ("reg_idx", C.c_void_p)]
+                ("beams", C.c_int32), ("max_new", C.c_int32), ("reg_idx", C.c_void_p),
+                ("priv_block_table", C.c_void_p), ("priv_pages_per_beam", C.c_int32), ("n_priv_pages", C.c_int32)]
 
 
 class EarnProj(C.Structure):
@@ -148,9 +149,11 @@ class Batch:
 
 
 def make_cache(k_shared=None, v_shared=None, block_table=None, pages_per_seq=0, n_pages=0, k_priv=None, v_priv=None,
-               lineage=None, beams=1, max_new=1, reg_idx=None) -> EarnCache:
+               lineage=None, beams=1, max_new=1, reg_idx=None, priv_block_table=None, priv_pages_per_beam=0,
+               n_priv_pages=0) -> EarnCache:
     return EarnCache(_ptr(k_shared), _ptr(v_shared), _ptr(block_table), pages_per_seq, n_pages, _ptr(k_priv),
-                     _ptr(v_priv), _ptr(lineage), beams, max_new, _ptr(reg_idx))
+                     _ptr(v_priv), _ptr(lineage), beams, max_new, _ptr(reg_idx), _ptr(priv_block_table),
+                     priv_pages_per_beam, n_priv_pages)
 
 
 def earn_version() -> int:

@@ -268,7 +268,7 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(DecodeArgs a) {
     const T* kn = reinterpret_cast<const T*>(a.k_new) + ((int64_t)j * a.Hkv + kvh) * D + lane * E;
     const T* vn = reinterpret_cast<const T*>(a.v_new) + ((int64_t)j * a.Hkv + kvh) * D + lane * E;
     if (gi == 0) {
-      int64_t dst = (((int64_t)j * a.max_new + t_new) * a.Hkv + kvh) * D + lane * E;
+      int64_t dst = (priv_row(a, j, t_new) * a.Hkv + kvh) * D + lane * E;
 #pragma unroll
       for (int e = 0; e < E; ++e) { kp[dst + e] = kn[e]; vp[dst + e] = vn[e]; }
     }
@@ -284,7 +284,7 @@ __global__ void __launch_bounds__(128) decode_merge_kernel(DecodeArgs a) {
       vr = reinterpret_cast<const T*>(a.v_new) + ((int64_t)j * a.Hkv + kvh) * D + lane * E;
     } else {
       int slab = a.lineage ? min(max(a.lineage[(int64_t)j * a.max_new + t], 0), a.batch * a.beams - 1) : j;
-      int64_t off = (((int64_t)slab * a.max_new + t) * a.Hkv + kvh) * D + lane * E;
+      int64_t off = (priv_row(a, slab, t) * a.Hkv + kvh) * D + lane * E;
       kr = kp + off;
       vr = vp + off;
     }

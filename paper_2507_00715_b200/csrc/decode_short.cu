@@ -94,7 +94,7 @@ __global__ void __launch_bounds__(NW * 32) decode_short_kernel(DecodeArgs a) {
         off = (j * a.Hkv + kvh) * D;
       } else {
         key = (int)(j * a.max_new + t);
-        off = ((j * a.max_new + t) * a.Hkv + kvh) * D;   // identity lineage; corrected behind the wait otherwise
+        off = ((j * a.max_new + t) * a.Hkv + kvh) * D;   // flat slabs, identity lineage; corrected behind the wait otherwise
       }
     }
     tab_off[p] = off;
@@ -155,11 +155,12 @@ __global__ void __launch_bounds__(NW * 32) decode_short_kernel(DecodeArgs a) {
     const int w = i / (2 * CH), c = i % (2 * CH), p = n_shared + w * step + step - 1;
     src = smem + (p >> 4) * G::STAGE_B + (c >= CH ? G::TILE_B : 0) + (p & 15) * G::PITCH + (c % CH) * 16;
     dst = reinterpret_cast<bf16*>(c >= CH ? a.v_priv : a.k_priv) +
-          ((((int64_t)b * W + w) * a.max_new + (step - 1)) * a.Hkv + kvh) * D + (c % CH) * 8;
+          (priv_row(a, (int64_t)b * W + w, step - 1) * a.Hkv + kvh) * D + (c % CH) * 8;
   };
   const uint8_t* app_src = nullptr;
   bf16* app_dst = nullptr;
-  if ((int)threadIdx.x < W * 2 * CH) app_piece(threadIdx.x, app_src, app_dst);
+  // (a page table of the private segment may have been written just ahead of this launch: it is read behind the wait)
+  if ((int)threadIdx.x < W * 2 * CH && a.priv_table == nullptr) app_piece(threadIdx.x, app_src, app_dst);
   {
     pin(app_src); pin(app_dst);
     pin(o_off0); pin(o_off1); pin(seen_bits);
@@ -188,10 +189,11 @@ __global__ void __launch_bounds__(NW * 32) decode_short_kernel(DecodeArgs a) {
       const int p = r_t + i * RPP;
       if (p_key[i] == -1) continue;
       int64_t off = p_off[i];
-      if (a.lineage != nullptr && p_key[i] >= 0) {   // the token lives in the slab of the beam that generated it
+      if ((a.lineage != nullptr || a.priv_table != nullptr) && p_key[i] >= 0) {
+        // the token lives in the slab of the beam that generated it, and possibly behind a page table
         const int t = p_key[i] % a.max_new;
-        const int64_t slab = min(max(a.lineage[p_key[i]], 0), a.batch * W - 1);
-        off = ((slab * a.max_new + t) * a.Hkv + kvh) * D + c_t * 8;
+        const int64_t slab = a.lineage != nullptr ? min(max(a.lineage[p_key[i]], 0), a.batch * W - 1) : p_key[i] / a.max_new;
+        off = (priv_row(a, slab, t) * a.Hkv + kvh) * D + c_t * 8;
       }
       const bool fresh = p_key[i] == -3;
       cp_async16(dst_of(p), (fresh ? knew : kpriv) + off);
@@ -204,7 +206,7 @@ __global__ void __launch_bounds__(NW * 32) decode_short_kernel(DecodeArgs a) {
 
   // ---- Eq. 4, append, from the tile in shared memory
   if (app_src != nullptr) *reinterpret_cast<uint4*>(app_dst) = *reinterpret_cast<const uint4*>(app_src);
-  for (int i = threadIdx.x + NT; i < W * 2 * CH; i += NT) {
+  for (int i = threadIdx.x + (a.priv_table == nullptr ? NT : 0); i < W * 2 * CH; i += NT) {
     app_piece(i, app_src, app_dst);
     *reinterpret_cast<uint4*>(app_dst) = *reinterpret_cast<const uint4*>(app_src);
   }

@@ -330,7 +330,7 @@ __device__ __forceinline__ int64_t private_row(const DecodeArgs& a, int b, int k
   int64_t slab = j;
   if (a.lineage) slab = min(max(a.lineage[j * a.max_new + t], 0), a.batch * a.beams - 1);
   which = 1;
-  return ((slab * a.max_new + t) * a.Hkv + kvh) * D;
+  return (priv_row(a, slab, t) * a.Hkv + kvh) * D;
 }
 
 // The three tensors a cache position can live in: 0 shared segment, 1 private segment, 2 this step's k_new / v_new.
@@ -379,7 +379,7 @@ struct AppendOne {
       const int c = tid % (2 * CH);
       is_v = c >= CH;
       piece = *reinterpret_cast<const uint4*>(reinterpret_cast<const bf16*>(is_v ? a.v_new : a.k_new) + (j * a.Hkv + rm.kvh) * D + (c % CH) * 8);
-      dst = ((j * a.max_new + (a.step - 1)) * a.Hkv + rm.kvh) * D + (c % CH) * 8;
+      dst = (priv_row(a, j, a.step - 1) * a.Hkv + rm.kvh) * D + (c % CH) * 8;
     }
   }
   __device__ __forceinline__ void store(const DecodeArgs& a) const {
@@ -404,7 +404,7 @@ __device__ __forceinline__ void append_new_rows(const DecodeArgs& a, const RowMa
     if (tid < n_items) {
       const int64_t j = (int64_t)rm.b * rm.W + w_first + tid / (2 * CH);
       const int c = tid % (2 * CH);
-      *reinterpret_cast<uint4*>((c < CH ? kp : vp) + ((j * a.max_new + (a.step - 1)) * a.Hkv + rm.kvh) * D + (c % CH) * 8) =
+      *reinterpret_cast<uint4*>((c < CH ? kp : vp) + (priv_row(a, j, a.step - 1) * a.Hkv + rm.kvh) * D + (c % CH) * 8) =
           *reinterpret_cast<const uint4*>((c < CH ? kn : vn) + (j * a.Hkv + rm.kvh) * D + (c % CH) * 8);
     }
     return;
@@ -426,7 +426,7 @@ __device__ __forceinline__ void append_new_rows(const DecodeArgs& a, const RowMa
       if (i < n_items) {
         const int64_t j = (int64_t)rm.b * rm.W + w_first + i / (2 * CH);
         const int c = i % (2 * CH);
-        *reinterpret_cast<uint4*>((c < CH ? kp : vp) + ((j * a.max_new + (a.step - 1)) * a.Hkv + rm.kvh) * D + (c % CH) * 8) = r[u];
+        *reinterpret_cast<uint4*>((c < CH ? kp : vp) + (priv_row(a, j, a.step - 1) * a.Hkv + rm.kvh) * D + (c % CH) * 8) = r[u];
       }
     }
   }

@@ -173,6 +173,9 @@ earn_status_t validate_decode(const earn_model_t* model, const earn_batch_t* bat
   if (layer < 0 || layer >= model->n_layers || cache == nullptr) return EARN_ERR_INVALID_ARG;
   if (cache->beams < 1 || cache->max_new < 1 || step < 1 || step > cache->max_new) return EARN_ERR_INVALID_ARG;
   if ((int64_t)batch->batch * cache->beams > 65535) return EARN_ERR_UNSUPPORTED;
+  if (cache->priv_block_table != nullptr &&
+      (cache->n_priv_pages < 1 || cache->priv_pages_per_beam < (cache->max_new + EARN_PAGE_TOKENS - 1) / EARN_PAGE_TOKENS))
+    return EARN_ERR_INVALID_ARG;
   if (batch->batch == 0) { *nothing_to_do = true; return EARN_OK; }
   if (layer < model->split_k) {
     if (!k_full || !v_full || !aligned16(k_full) || !aligned16(v_full)) return EARN_ERR_INVALID_ARG;
@@ -368,6 +371,7 @@ earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* ba
   }
   a.cu_seqlens = batch->cu_seqlens;
   a.k_priv = cache->k_priv; a.v_priv = cache->v_priv; a.lineage = cache->lineage;
+  a.priv_table = cache->priv_block_table; a.priv_pages_per_beam = cache->priv_pages_per_beam; a.n_priv_pages = cache->n_priv_pages;
   a.plan = make_decode_plan(*model, *batch, cache->beams,
                             early ? batch->max_seqlen : batch->n_head_reg + batch->n_tail_reg);
   const size_t tickets_at = kStatusBytes + prefill_plan_bytes(*batch);

@@ -138,6 +138,8 @@ struct DecodeArgs {
   const int32_t* cu_seqlens;   // device, for the shared length of a packed source
   void *k_priv, *v_priv;
   const int32_t* lineage;
+  const int32_t* priv_table;   // page table of the private segment [B*W, priv_pages_per_beam], or null: flat slabs
+  int priv_pages_per_beam, n_priv_pages;
   float* part_o;               // [B, Hkv, n_splits, rows_pad, D]
   float* part_lse;             // [B, Hkv, n_splits, rows_pad]  (log2 domain)
   int32_t* tickets;            // [B, Hkv, row_tiles], zero between launches: which split finished last
@@ -152,6 +154,14 @@ struct DecodeArgs {
   // after the key loop
   int trigger_early;
 };
+// Row of the private (generated-token) segment that holds token t of slab `slab` (the beam that generated it): row
+// slab * max_new + t of the flat layout, or, behind a page table, slot t % 16 of page priv_table[slab][t / 16].
+__device__ __forceinline__ int64_t priv_row(const DecodeArgs& a, int64_t slab, int t) {
+  if (a.priv_table == nullptr) return slab * a.max_new + t;
+  int page = a.priv_table[slab * a.priv_pages_per_beam + t / EARN_PAGE_TOKENS];
+  page = min(max(page, 0), a.n_priv_pages - 1);   // a corrupt table reads or writes a wrong page, never outside the cache
+  return (int64_t)page * EARN_PAGE_TOKENS + t % EARN_PAGE_TOKENS;
+}
 cudaError_t launch_decode_simt(const DecodeArgs& a, cudaStream_t st);   // fp32 debug path
 // bf16: cp.async ring + mma.sync; max_shared_len = longest shared segment of the batch (picks the ring depth)
 cudaError_t launch_decode_mma(const DecodeArgs& a, int max_shared_len, cudaStream_t st);

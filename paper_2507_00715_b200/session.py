@@ -20,7 +20,8 @@ class EarnSession:
 
     def __init__(self, n_layers: int, split_k: int, n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: torch.dtype,
                  cu_seqlens: np.ndarray, r_head: int, r_tail: int, beams: int = 1, max_new: int = 1,
-                 softmax_scale: float = 0.0, device="cuda", paged_shuffle_seed: Optional[int] = None):
+                 softmax_scale: float = 0.0, device="cuda", paged_shuffle_seed: Optional[int] = None,
+                 paged_private_seed: Optional[int] = None):
         self.device = torch.device(device)
         self.dtype = dtype
         self.model = B.make_model(n_layers, split_k, n_q_heads, n_kv_heads, head_dim, dtype, softmax_scale)
@@ -43,12 +44,23 @@ class EarnSession:
         self.k_full: List[Optional[torch.Tensor]] = [None] * n_layers
         self.v_full: List[Optional[torch.Tensor]] = [None] * n_layers
         self.k_priv, self.v_priv = [], []
+        # the private (generated-token) segment: flat slabs, or pages behind a scattered table (one table for all layers)
+        self.priv_table, self.priv_pages_per_beam, self.n_priv_pages = None, 0, 0
+        if paged_private_seed is not None:
+            self.priv_pages_per_beam = -(-self.max_new // B.PAGE_TOKENS)
+            self.n_priv_pages = max(1, nb * beams * self.priv_pages_per_beam)
+            perm = np.random.Generator(np.random.Philox(paged_private_seed)).permutation(self.n_priv_pages)
+            self.priv_table = torch.from_numpy(perm.astype(np.int32).reshape(nb * beams, self.priv_pages_per_beam)).to(self.device)
         for layer in range(n_layers):
             if layer >= split_k:
                 self.k_shared[layer] = torch.zeros(self.n_pages, B.PAGE_TOKENS, n_kv_heads, head_dim, **kw)
                 self.v_shared[layer] = torch.zeros(self.n_pages, B.PAGE_TOKENS, n_kv_heads, head_dim, **kw)
-            self.k_priv.append(torch.zeros(nb * beams, self.max_new, n_kv_heads, head_dim, **kw))
-            self.v_priv.append(torch.zeros(nb * beams, self.max_new, n_kv_heads, head_dim, **kw))
+            if self.priv_table is not None:
+                self.k_priv.append(torch.zeros(self.n_priv_pages, B.PAGE_TOKENS, n_kv_heads, head_dim, **kw))
+                self.v_priv.append(torch.zeros(self.n_priv_pages, B.PAGE_TOKENS, n_kv_heads, head_dim, **kw))
+            else:
+                self.k_priv.append(torch.zeros(nb * beams, self.max_new, n_kv_heads, head_dim, **kw))
+                self.v_priv.append(torch.zeros(nb * beams, self.max_new, n_kv_heads, head_dim, **kw))
         self.reg_idx = torch.zeros(nb, max(R, 1), dtype=torch.int32, device=self.device)
         self.lineage = [torch.zeros(nb * beams, self.max_new, dtype=torch.int32, device=self.device) for _ in range(2)]
         self.lineage_cur: Optional[int] = None      # None = identity table
@@ -61,7 +73,7 @@ class EarnSession:
         lin = None if self.lineage_cur is None else self.lineage[self.lineage_cur]
         return B.make_cache(self.k_shared[layer], self.v_shared[layer], self.block_table, self.pages_per_seq,
                             self.n_pages, self.k_priv[layer], self.v_priv[layer], lin, self.beams, self.max_new,
-                            self.reg_idx)
+                            self.reg_idx, self.priv_table, self.priv_pages_per_beam, self.n_priv_pages)
 
     # ---- prefill
     def prefill_layer(self, layer: int, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,

@@ -101,6 +101,10 @@ def test_host_validation_compact_register_decode(lib):
     assert dec(2, 5) == B.EARN_ERR_INVALID_ARG                    # beyond max_new
     assert dec(2, 1, ws_bytes=256) == B.EARN_ERR_WORKSPACE
     assert dec(4, 1) == B.EARN_ERR_INVALID_ARG
+    # a paged private segment: 20 generated tokens need two pages per beam
+    paged = B.make_cache(0x1000, 0x1000, None, 2, 4, 0x1000, 0x1000, None, 1, 20, None, 0x7000, 1, 8)
+    assert dec(2, 1, cache=paged) == B.EARN_ERR_INVALID_ARG
+    assert dec(2, 1, cache=B.make_cache(0x1000, 0x1000, None, 2, 4, 0x1000, 0x1000, None, 1, 20, None, 0x7000, 2, 0)) == B.EARN_ERR_INVALID_ARG
 
     assert lib.earn_beam_reparent(2, 3, 4, 2, 0x1000, 0x2000, 0x2000, None) == B.EARN_ERR_INVALID_ARG   # aliasing tables
     assert lib.earn_beam_reparent(2, 3, 4, 5, 0x1000, None, 0x2000, None) == B.EARN_ERR_INVALID_ARG

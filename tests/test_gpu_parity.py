@@ -186,3 +186,15 @@ def test_one_token_sequences_among_long_ones():
     of a single valid row, compaction keeps the only token, decode sees a one-key prompt cache."""
     run_workload_and_compare(BASE.replace(seed=29, lens=(1, 300, 2, 129, 1), batch=5, r_head=1, r_tail=0, beams=2,
                                           decode_steps=2))
+
+
+@pytest.mark.parametrize("shape", ["one_row_tile", "several_row_tiles", "fp32", "short_list_head_dim_64"])
+def test_private_segment_behind_a_page_table(shape):
+    """The generated tokens live in scattered 16-token pages (one table for every layer) instead of flat slabs: 18
+    decode steps cross a page boundary, beams are re-parented every step, every decode kernel family takes a turn."""
+    kw = {"one_row_tile": dict(n_q_heads=4, n_kv_heads=2, beams=3),                 # streaming + short-list kernels
+          "several_row_tiles": dict(n_q_heads=8, n_kv_heads=2, beams=5),             # 20 query rows per kv head
+          "fp32": dict(dtype="f32", n_q_heads=4, n_kv_heads=2, beams=2, head_dim=64),
+          "short_list_head_dim_64": dict(head_dim=64, n_q_heads=4, n_kv_heads=2, beams=2)}[shape]
+    w = BASE.replace(seed=23, lens=(90, 40), batch=2, n_layers=2, split_k=1, r_head=4, r_tail=4, decode_steps=18, **kw)
+    run_workload_and_compare(w, check_lse=False, paged_private_seed=9, paged_shuffle_seed=3)
