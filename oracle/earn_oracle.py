@@ -26,6 +26,11 @@ What pins each function (see tests/test_oracle_pins.py):
                           "project every row then gather" = "gather then project" (Eq. 2 acts per token)
   rope_tables           : closed-form angles (D = 8, theta = 10000: 1, 0.1, 0.01, 0.001 rad per position)
   attention_scores, sparsity, sinks : the scalar definitions of Eq. 14-15 by hand
+  causal_attention_grad : central finite differences of a scalar loss through causal_attention; torch autograd (fp64)
+                          through a library SDPA call (with k = N training is ordinary causal attention)
+  participating_attention(_grad), participating_indices : autograd through a dense full-length attention whose mask
+                          is the training rule itself (keys restricted to the participating set) gives the same outputs
+                          on the participating rows and the same gradients, zero on every prompt row
   beam_topk             : python's sorted() on (score, index) tuples; hand-made cases (a dominant beam, exact ties,
                           the first step with one live beam); greedy decoding (one beam) = argmax
 Attention values have no printed worked example in the paper, so beyond those
@@ -311,6 +316,77 @@ class DecodeState:
     def entries(self, b: int) -> int:
         """KV entries one beam of sequence b reads in this layer (per kv head)."""
         return self.shared_k[b].shape[0] + len(self.priv_k[b * self.beams])
+
+
+# --------------------------------------------------------------------------
+# Section 3.2, "Training": the sample is X ++ Y = [R_prefix; Prompt; R_suffix; Y] (Eq. 5-6, Y the target identifier,
+# teacher-forced), the loss of Eq. 7 is taken on Y, and the attention differs from ordinary finetuning only in who
+# takes part: layers l <= k (1-indexed) all tokens, layers l > k only register and generated (target) tokens.
+# Forward is Eq. 3 under that rule; backward is the chain rule through Eq. 3:
+#   P = softmax(S), O = P V   =>   dV = P^T dO,  dP = dO V^T,  dS = P o (dP - rowsum(dO o O)),  dQ = dS K c,  dK = dS^T Q c
+# with c the logit scale.  Query heads of a group add their dK, dV into the kv head they share.
+# --------------------------------------------------------------------------
+def participating_indices(seqlens: Sequence[int], r_head: int, r_tail: int, n_target: int) -> np.ndarray:
+    """Positions of the tokens that take part in a layer l > k of a TRAINING sequence of length L_b (targets
+    included): the r_head prefix registers, the r_tail suffix registers and the n_target target tokens, in order,
+    int32 [B, r_head + r_tail + n_target].  The suffix registers and the targets are the last r_tail + n_target rows."""
+    return register_indices(seqlens, r_head, r_tail + n_target)
+
+
+def causal_attention_grad(q, k, v, cu_seqlens, d_o, scale: Optional[float] = None):
+    """Gradients of causal_attention's output with respect to q, k, v for an upstream gradient d_o [total,Hq,D]:
+    returns (dq [total,Hq,D], dk [total,Hkv,D], dv [total,Hkv,D]), float64."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    d_o = np.asarray(d_o, dtype=np.float64)
+    total, hq, d = q.shape
+    g = hq // k.shape[1]
+    sc = _scale(d, scale)
+    dq, dk, dv = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v)
+    for b in range(len(cu_seqlens) - 1):
+        lo, hi = int(cu_seqlens[b]), int(cu_seqlens[b + 1])
+        n = hi - lo
+        if n == 0:
+            continue
+        allowed = np.tril(np.ones((n, n), dtype=bool))
+        for h in range(hq):
+            kh = h // g
+            s = np.where(allowed, (q[lo:hi, h, :] @ k[lo:hi, kh, :].T) * sc, -np.inf)
+            p, _ = _softmax_rows(s)
+            o = p @ v[lo:hi, kh, :]
+            go = d_o[lo:hi, h, :]
+            dv[lo:hi, kh, :] += p.T @ go
+            dp = go @ v[lo:hi, kh, :].T
+            ds = p * (dp - np.sum(go * o, axis=1, keepdims=True))
+            dq[lo:hi, h, :] = (ds @ k[lo:hi, kh, :]) * sc
+            dk[lo:hi, kh, :] += (ds.T @ q[lo:hi, h, :]) * sc
+    return dq, dk, dv
+
+
+def participating_attention(q_p, k_p, v_p, scale: Optional[float] = None):
+    """A layer l > k of a training sample on the rows that take part (gathered in order [prefix; suffix; targets]):
+    causal attention among them.  q_p [B,P,Hq,D], k_p, v_p [B,P,Hkv,D] -> (O [B,P,Hq,D], LSE [B,Hq,P]) float64."""
+    b_, p_, hq, d = q_p.shape
+    if p_ == 0:
+        return np.zeros((b_, 0, hq, d)), np.zeros((b_, hq, 0))
+    cu = np.arange(b_ + 1, dtype=np.int64) * p_
+    o, lse = causal_attention(np.asarray(q_p).reshape(b_ * p_, hq, d), np.asarray(k_p).reshape(b_ * p_, -1, d),
+                              np.asarray(v_p).reshape(b_ * p_, -1, d), cu, scale)
+    return o.reshape(b_, p_, hq, d), lse.reshape(hq, b_, p_).transpose(1, 0, 2).copy()
+
+
+def participating_attention_grad(q_p, k_p, v_p, d_o_p, scale: Optional[float] = None):
+    """Backward of participating_attention: (dq_p, dk_p, dv_p), shapes of the inputs, float64."""
+    b_, p_, hq, d = q_p.shape
+    hkv = k_p.shape[2]
+    if p_ == 0:
+        return np.zeros((b_, 0, hq, d)), np.zeros((b_, 0, hkv, d)), np.zeros((b_, 0, hkv, d))
+    cu = np.arange(b_ + 1, dtype=np.int64) * p_
+    dq, dk, dv = causal_attention_grad(np.asarray(q_p).reshape(b_ * p_, hq, d), np.asarray(k_p).reshape(b_ * p_, hkv, d),
+                                       np.asarray(v_p).reshape(b_ * p_, hkv, d), cu,
+                                       np.asarray(d_o_p).reshape(b_ * p_, hq, d), scale)
+    return dq.reshape(b_, p_, hq, d), dk.reshape(b_, p_, hkv, d), dv.reshape(b_, p_, hkv, d)
 
 
 # --------------------------------------------------------------------------

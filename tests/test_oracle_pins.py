@@ -485,3 +485,89 @@ def test_beam_topk_matches_sorted_tuples_and_hand_cases():
     assert not p5.any() and list(t5) == list(lp5.argmax(axis=1)) and np.array_equal(s5, lp5.max(axis=1))
     with pytest.raises(ValueError):
         orc.beam_topk(np.zeros((4, 3), np.float32), np.zeros(4, np.float32), 4, n_live=1)   # 3 candidates for 4 slots
+
+
+# ---------------------------------------------------------------- training (Section 3.2 "Training", Eq. 7)
+def _torch_masked_attention(q, k, v, allowed):
+    """Dense attention of one sequence in torch fp64 under an explicit boolean mask [n, n] (library softmax / matmul),
+    GQA heads expanded by hand: q [n,Hq,D], k, v [n,Hkv,D] tensors that require grad."""
+    hq, hkv, d = q.shape[1], k.shape[1], q.shape[2]
+    kk = k.repeat_interleave(hq // hkv, dim=1)
+    vv = v.repeat_interleave(hq // hkv, dim=1)
+    s = torch.einsum("ihd,jhd->hij", q, kk) / math.sqrt(d)
+    s = s.masked_fill(~allowed[None], float("-inf"))
+    return torch.einsum("hij,jhd->ihd", torch.softmax(s, dim=-1), vv)
+
+
+def test_causal_attention_grad_matches_finite_differences_and_autograd():
+    rng = np.random.default_rng(14)
+    cu = np.array([0, 5, 6, 13])
+    q, k, v = rand_qkv(rng, 13, 4, 2, 3)
+    go = rng.standard_normal(q.shape)
+    dq, dk, dv = orc.causal_attention_grad(q, k, v, cu, go)
+    loss = lambda q_, k_, v_: float(np.sum(orc.causal_attention(q_, k_, v_, cu)[0] * go))   # noqa: E731
+    eps = 1e-6
+    for arr, grad, which in ((q, dq, 0), (k, dk, 1), (v, dv, 2)):
+        for _ in range(12):                                    # sampled coordinates, central differences
+            i = tuple(int(rng.integers(0, n)) for n in arr.shape)
+            hi, lo = arr.copy(), arr.copy()
+            hi[i] += eps
+            lo[i] -= eps
+            args_hi = [q, k, v]
+            args_lo = [q, k, v]
+            args_hi[which], args_lo[which] = hi, lo
+            fd = (loss(*args_hi) - loss(*args_lo)) / (2 * eps)
+            assert abs(fd - grad[i]) < 1e-7, (which, i, fd, grad[i])
+    # k = N: every layer is ordinary causal attention; torch autograd through the library SDPA, sequence by sequence
+    for b in range(3):
+        sl = slice(cu[b], cu[b + 1])
+        tq, tk, tv = (torch.from_numpy(x[sl]).clone().requires_grad_(True) for x in (q, k, v))
+        o = torch.nn.functional.scaled_dot_product_attention(
+            tq.permute(1, 0, 2)[None], tk.permute(1, 0, 2)[None].repeat_interleave(2, dim=1),
+            tv.permute(1, 0, 2)[None].repeat_interleave(2, dim=1), is_causal=True)[0].permute(1, 0, 2)
+        (o * torch.from_numpy(go[sl])).sum().backward()
+        np.testing.assert_allclose(dq[sl], tq.grad.numpy(), atol=1e-12)
+        np.testing.assert_allclose(dk[sl], tk.grad.numpy(), atol=1e-12)
+        np.testing.assert_allclose(dv[sl], tv.grad.numpy(), atol=1e-12)
+
+
+@pytest.mark.parametrize("rh,rt,nt", [(2, 1, 3), (0, 2, 4), (1, 0, 1), (2, 2, 0)])
+def test_training_rule_for_layers_after_the_split(rh, rt, nt):
+    """Layers l > k of a training sample: only register and target tokens take part.  Stated as a mask on a dense
+    full-length attention (keys restricted to the participating set, causal) and differentiated by torch autograd, it
+    gives on the participating rows what the oracle computes on the gathered rows, the same gradients there, and no
+    gradient at all on the prompt rows."""
+    rng = np.random.default_rng(15)
+    lens = [11, rh + rt + nt + 1, rh + rt + nt]
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    q, k, v = rand_qkv(rng, cu[-1], 4, 2, 5)
+    idx = orc.participating_indices(lens, rh, rt, nt)
+    P = rh + rt + nt
+    for b, L in enumerate(lens):                              # the layout [prefix; ...; suffix; targets] by hand
+        assert list(idx[b]) == list(range(rh)) + list(range(L - nt - rt, L))
+    q_p, k_p, v_p = orc.compact(q, cu, idx), orc.compact(k, cu, idx), orc.compact(v, cu, idx)
+    go_p = rng.standard_normal(q_p.shape)
+    o_p, lse_p = orc.participating_attention(q_p, k_p, v_p)
+    dq_p, dk_p, dv_p = orc.participating_attention_grad(q_p, k_p, v_p, go_p)
+    assert o_p.shape == (3, P, 4, 5) and lse_p.shape == (3, 4, P)
+    for b, L in enumerate(lens):
+        sl = slice(cu[b], cu[b + 1])
+        tq, tk, tv = (torch.from_numpy(x[sl]).clone().requires_grad_(True) for x in (q, k, v))
+        part = torch.zeros(L, dtype=torch.bool)
+        part[torch.from_numpy(idx[b]).long()] = True
+        allowed = torch.tril(torch.ones(L, L, dtype=torch.bool)) & part[None, :]
+        allowed |= torch.eye(L, dtype=torch.bool) & ~part[:, None]       # prompt rows (unused) keep one key: no empty row
+        o = _torch_masked_attention(tq, tk, tv, allowed)
+        rows = torch.from_numpy(idx[b]).long()
+        np.testing.assert_allclose(o[rows].detach().numpy(), o_p[b], atol=1e-12)
+        (o[rows] * torch.from_numpy(go_p[b])).sum().backward()           # the loss sees the participating rows only
+        for grad_p, t in ((dq_p, tq), (dk_p, tk), (dv_p, tv)):
+            full = t.grad.numpy()
+            np.testing.assert_allclose(full[idx[b]], grad_p[b], atol=1e-12)
+            rest = np.ones(L, bool)
+            rest[idx[b]] = False
+            assert not full[rest].any()                                    # removed tokens receive no gradient
+    # LSE of one row by hand
+    b, m, h = 0, P - 1, 3
+    logits = [float(q_p[b, m, h] @ k_p[b, j, 1]) / math.sqrt(5) for j in range(P)]
+    assert abs(lse_p[b, h, m] - math.log(math.fsum(math.exp(x) for x in logits))) < 1e-12
