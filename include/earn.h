@@ -222,6 +222,33 @@ earn_status_t earn_beam_reparent(int32_t batch, int32_t beams, int32_t max_new, 
                                  const int32_t* parent, const int32_t* lineage_in_or_null,
                                  int32_t* lineage_out, earn_stream_t stream);
 
+/* Training-time attention (Section 3.2 "Training"; the loss of Eq. 7 is taken on the target identifier Y).  A training
+ * sample is the sequence [prefix registers; prompt; suffix registers; Y] with the n_target tokens of Y teacher-forced at
+ * its end; `batch` describes those sequences (every L_b counts the targets, L_b >= r_h + r_t + n_target).  The paper
+ * changes one thing against ordinary finetuning: who takes part in the attention of a layer.
+ *   layer <  k : every token (ordinary causal attention, Eq. 3).  q, o, d_o, dq: device [total_tokens, Hq, D];
+ *                k, v, dk, dv: device [total_tokens, Hkv, D]; lse: device fp32 [Hq, total_tokens].
+ *   layer >= k : only register and target tokens, P = r_h + r_t + n_target per sequence, in the order [prefix; suffix;
+ *                targets] (the suffix registers and the targets are the last r_t + n_target rows of a sequence).  The
+ *                prompt rows were removed from the hidden state at layer k, so the tensors hold the participating rows
+ *                only: q, o, d_o, dq: device [B, P, Hq, D]; k, v, dk, dv: device [B, P, Hkv, D]; lse: fp32 [B, Hq, P];
+ *                causal attention among them.  Removed tokens have no output and receive no gradient in these layers.
+ * Forward writes o and lse (natural-log softmax denominators; required: the backward reads them).  Backward takes the
+ * forward's inputs and outputs and the upstream gradient d_o and writes
+ *   dV = P^T dO,   dS = P o (dO V^T - rowsum(dO o O)),   dQ = dS K * scale,   dK = dS^T Q * scale,
+ * the query heads of a group adding into the kv head they share.  fp32 arithmetic, one rounding to the model dtype.
+ * workspace: at least earn_train_workspace_bytes(model, batch) bytes, zeroed once by earn_workspace_init.
+ * Errors: layer outside [0, N), n_target < 0, a sequence shorter than r_h + r_t + n_target, NULL or misaligned tensors
+ * -> INVALID_ARG; workspace NULL / too small -> WORKSPACE. */
+size_t earn_train_workspace_bytes(const earn_model_t* model, const earn_batch_t* batch);
+earn_status_t earn_train_attn_fwd(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, int32_t n_target,
+                                  const void* q, const void* k, const void* v, void* o, float* lse,
+                                  void* workspace, size_t workspace_bytes, earn_stream_t stream);
+earn_status_t earn_train_attn_bwd(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, int32_t n_target,
+                                  const void* q, const void* k, const void* v, const void* o, const float* lse,
+                                  const void* d_o, void* dq, void* dk, void* dv,
+                                  void* workspace, size_t workspace_bytes, earn_stream_t stream);
+
 /* Beam selection between decode steps (Appendix A.3: identifiers are generated by beam search, beam size 20; the paper
  * gives the beam size only, the rule is that of ordinary beam search).  For every sequence, of the n_live * vocab
  * continuations (beam w < n_live, token v), scored beam_scores[b*W + w] + logprobs[b*W + w][v] in fp32, the W best

@@ -70,6 +70,12 @@ SYMBOLS = {
                                           C.c_void_p]),
     "earn_beam_reparent": (C.c_int, [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                      C.c_void_p, C.c_void_p]),
+    "earn_train_workspace_bytes": (C.c_size_t, [C.POINTER(EarnModel), C.POINTER(EarnBatch)]),
+    "earn_train_attn_fwd": (C.c_int, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "earn_train_attn_bwd": (C.c_int, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                      C.c_void_p, C.c_size_t, C.c_void_p]),
     "earn_beam_topk_workspace_bytes": (C.c_size_t, [C.c_int32, C.c_int32, C.c_int32]),
     "earn_beam_topk": (C.c_int, [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                  C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -254,3 +260,20 @@ def earn_beam_topk(batch: int, beams: int, n_live: int, vocab: int, logprobs, be
     p, n = _ws(workspace)
     _check(lib().earn_beam_topk(batch, beams, n_live, vocab, _ptr(logprobs), _ptr(beam_scores), _ptr(parent), _ptr(token),
                                 _ptr(new_scores), p, n, _stream()), "earn_beam_topk")
+
+
+def earn_train_workspace_bytes(model: EarnModel, batch: Batch) -> int:
+    return lib().earn_train_workspace_bytes(C.byref(model), C.byref(batch.c))
+
+
+def earn_train_attn_fwd(model, batch: Batch, layer, n_target, q, k, v, o, lse, workspace) -> None:
+    p, n = _ws(workspace)
+    _check(lib().earn_train_attn_fwd(C.byref(model), C.byref(batch.c), layer, n_target, _ptr(q), _ptr(k), _ptr(v), _ptr(o),
+                                     _ptr(lse), p, n, _stream()), "earn_train_attn_fwd")
+
+
+def earn_train_attn_bwd(model, batch: Batch, layer, n_target, q, k, v, o, lse, d_o, dq, dk, dv, workspace) -> None:
+    p, n = _ws(workspace)
+    _check(lib().earn_train_attn_bwd(C.byref(model), C.byref(batch.c), layer, n_target, _ptr(q), _ptr(k), _ptr(v), _ptr(o),
+                                     _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv), p, n, _stream()),
+           "earn_train_attn_bwd")

@@ -418,6 +418,93 @@ earn_status_t earn_beam_reparent(int32_t batch, int32_t beams, int32_t max_new, 
   return ok ? EARN_OK : EARN_ERR_CUDA;
 }
 
+static size_t train_scratch_bytes(const earn_model_t* m, const earn_batch_t* b) {
+  return round_up(sizeof(float) * (size_t)m->n_q_heads * (size_t)b->total_tokens, 256);   // one [Hq, total] fp32 array
+}
+
+size_t earn_train_workspace_bytes(const earn_model_t* model, const earn_batch_t* batch) {
+  if (check_model(model) != EARN_OK || check_batch(batch) != EARN_OK) return kStatusBytes;
+  // status block | plan of the forward (and, afterwards, of the backward) | delta | LSE in the log2 domain
+  return kStatusBytes + prefill_plan_bytes(*batch) + 2 * train_scratch_bytes(model, batch) + 256;
+}
+
+// shared argument checks of the two training calls; fills the kernel arguments
+static earn_status_t train_setup(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, int32_t n_target,
+                                 const void* q, const void* k, const void* v, const void* o, const float* lse,
+                                 void* workspace, size_t workspace_bytes, TrainArgs* a, bool* nothing_to_do) {
+  *nothing_to_do = false;
+  earn_status_t s = check_model(model);
+  if (s != EARN_OK) return s;
+  s = check_batch(batch);
+  if (s != EARN_OK) return s;
+  if (layer < 0 || layer >= model->n_layers || n_target < 0) return EARN_ERR_INVALID_ARG;
+  const int P = batch->n_head_reg + batch->n_tail_reg + n_target;
+  for (int i = 0; i < batch->batch; ++i)
+    if (batch->cu_seqlens_host[i + 1] - batch->cu_seqlens_host[i] < P) return EARN_ERR_INVALID_ARG;
+  const bool full = layer < model->split_k;
+  if (batch->batch == 0 || (full ? batch->total_tokens == 0 : P == 0)) { *nothing_to_do = true; return EARN_OK; }
+  if (!q || !k || !v || !o || !lse) return EARN_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(lse)) return EARN_ERR_INVALID_ARG;
+  if (workspace == nullptr || !aligned16(workspace) || workspace_bytes < earn_train_workspace_bytes(model, batch))
+    return EARN_ERR_WORKSPACE;
+  *a = TrainArgs{};
+  a->q = q; a->k = k; a->v = v; a->o = o; a->lse = const_cast<float*>(lse);
+  a->batch = batch->batch; a->Hq = model->n_q_heads; a->Hkv = model->n_kv_heads; a->D = model->head_dim;
+  a->dtype = model->dtype; a->scale = scale_of(model);
+  if (full) {
+    a->cu_seqlens = batch->cu_seqlens; a->total = batch->total_tokens; a->max_seqlen = batch->max_seqlen;
+  } else {
+    a->cu_seqlens = nullptr; a->uniform_len = P; a->total = batch->batch * P; a->max_seqlen = P;
+  }
+  char* ws = reinterpret_cast<char*>(workspace);
+  a->status = reinterpret_cast<int32_t*>(ws);
+  a->delta = reinterpret_cast<float*>(ws + kStatusBytes + prefill_plan_bytes(*batch));
+  a->lse2 = reinterpret_cast<float*>(ws + kStatusBytes + prefill_plan_bytes(*batch) + train_scratch_bytes(model, batch));
+  return EARN_OK;
+}
+
+earn_status_t earn_train_attn_fwd(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, int32_t n_target,
+                                  const void* q, const void* k, const void* v, void* o, float* lse, void* workspace,
+                                  size_t workspace_bytes, earn_stream_t stream) {
+  TrainArgs a;
+  bool nothing = false;
+  earn_status_t s = train_setup(model, batch, layer, n_target, q, k, v, o, lse, workspace, workspace_bytes, &a, &nothing);
+  if (s != EARN_OK || nothing) return s;
+  a.out_o = o;
+  note_call(stream, CALL_UNKNOWN);
+  if (layer < model->split_k) {
+    // ordinary causal attention: the prefill kernel, with the softmax denominators kept for the backward
+    PrefillArgs p{};
+    p.q = q; p.k = k; p.v = v; p.o = o; p.lse = lse; p.cu_seqlens = batch->cu_seqlens;
+    p.batch = batch->batch; p.max_seqlen = batch->max_seqlen;
+    p.Hq = a.Hq; p.Hkv = a.Hkv; p.D = a.D; p.dtype = a.dtype; p.scale = a.scale;
+    if (prefill_tc_supported(p, batch->total_tokens))
+      return launch_prefill_tc(p, batch->total_tokens,
+                               prefill_plan_entries(*batch, prefill_rows_per_entry(model->n_q_heads, model->n_kv_heads)),
+                               reinterpret_cast<char*>(workspace) + kStatusBytes, a.status,
+                               (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+  }
+  return launch_train_fwd_simt(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+}
+
+earn_status_t earn_train_attn_bwd(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, int32_t n_target,
+                                  const void* q, const void* k, const void* v, const void* o, const float* lse,
+                                  const void* d_o, void* dq, void* dk, void* dv, void* workspace, size_t workspace_bytes,
+                                  earn_stream_t stream) {
+  TrainArgs a;
+  bool nothing = false;
+  earn_status_t s = train_setup(model, batch, layer, n_target, q, k, v, o, lse, workspace, workspace_bytes, &a, &nothing);
+  if (s != EARN_OK || nothing) return s;
+  if (!d_o || !dq || !dk || !dv || !aligned16(d_o) || !aligned16(dq) || !aligned16(dk) || !aligned16(dv))
+    return EARN_ERR_INVALID_ARG;
+  a.d_o = d_o; a.dq = dq; a.dk = dk; a.dv = dv;
+  note_call(stream, CALL_UNKNOWN);
+  if (layer < model->split_k && train_bwd_tc_supported(a))
+    return launch_train_bwd_tc(a, *batch, reinterpret_cast<char*>(workspace) + kStatusBytes, (cudaStream_t)stream) == cudaSuccess
+               ? EARN_OK : EARN_ERR_CUDA;
+  return launch_train_bwd_simt(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+}
+
 size_t earn_beam_topk_workspace_bytes(int32_t batch, int32_t beams, int32_t vocab) {
   if (batch < 0 || beams < 1 || beams > 32 || vocab < 1 || !beam_topk_supported(beams, vocab)) return 256;
   return beam_topk_workspace(batch, beams, vocab);

@@ -200,6 +200,28 @@ cudaError_t launch_register_qkv(const RegisterQkvArgs& a, cudaStream_t st);
 cudaError_t launch_beam_reparent(int batch, int beams, int max_new, int step, const int32_t* parent,
                                  const int32_t* lineage_in, int32_t* lineage_out, cudaStream_t st);
 
+// training-time attention (Section 3.2 "Training"): forward with LSE and backward, over packed sequences
+// (cu_seqlens) or over the gathered participating rows of the layers after the split (uniform_len rows per sequence)
+struct TrainArgs {
+  const void *q, *k, *v;       // [rows, Hq, D], [rows, Hkv, D]
+  const void* o;               // backward: the forward's output
+  const void* d_o;             // backward: upstream gradient, shape of o
+  void* out_o;                 // forward: output
+  float* lse;                  // natural-log softmax denominators: [Hq, total] (packed) or [B, Hq, P] (uniform); forward writes, backward reads
+  void *dq, *dk, *dv;          // backward outputs, shapes of q, k, v
+  const int32_t* cu_seqlens;   // device [B+1], or null: sequence b is rows b * uniform_len .. + uniform_len
+  int uniform_len;
+  int batch, total, max_seqlen, Hq, Hkv, D, dtype;
+  float scale;
+  float* delta;                // scratch fp32 [Hq, total]: rowsum(dO o O) (tensor-core path)
+  float* lse2;                 // scratch fp32 [Hq, total]: LSE in the log2 domain (tensor-core path)
+  int32_t* status;
+};
+cudaError_t launch_train_fwd_simt(const TrainArgs& a, cudaStream_t st);
+cudaError_t launch_train_bwd_simt(const TrainArgs& a, cudaStream_t st);
+bool train_bwd_tc_supported(const TrainArgs& a);   // bf16, head_dim 128, packed sequences
+cudaError_t launch_train_bwd_tc(const TrainArgs& a, const earn_batch_t& b, void* plan, cudaStream_t st);
+
 // beam selection (top W of n_live * vocab continuations per sequence)
 bool beam_topk_supported(int beams, int vocab);
 size_t beam_topk_workspace(int batch, int beams, int vocab);

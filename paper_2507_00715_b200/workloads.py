@@ -102,7 +102,7 @@ CONFIGS["paper_gqa"] = Workload("paper_gqa", batch=48, n_layers=28, split_k=7, n
 LONG_SPLIT_SWEEP = (2, 4, 8, 16)
 
 _TAG = {"q": 1, "k": 2, "v": 3, "dq": 4, "dk": 5, "dv": 6, "len": 7, "u": 8, "parent": 9, "x": 10, "wn": 11, "wqkv": 12,
-        "logits": 13}
+        "logits": 13, "go": 14}
 
 
 def _seed_for(w: Workload, tag: str, layer: int = 0, step: int = 0) -> int:
@@ -214,3 +214,9 @@ def beam_logprobs(w: Workload, step: int, vocab: int, device="cpu", allowed: int
             keep[r, torch.randperm(vocab, generator=g)[:allowed]] = True
         logits = torch.where(keep.to(device), logits, torch.full_like(logits, float("-inf")))
     return torch.log_softmax(logits, dim=-1)
+
+
+def upstream_grad(w: Workload, layer: int, shape, device="cpu") -> torch.Tensor:
+    """Gradient of the loss with respect to an attention output of the given shape, ~ N(0,1), in the workload dtype
+    (there is no loss here to produce it)."""
+    return _randn(tuple(shape), _seed_for(w, "go", layer), device).to(w.torch_dtype)
