@@ -116,6 +116,9 @@ cudaError_t launch_prefill_simt(const PrefillArgs& a, cudaStream_t st);
 bool prefill_tc_supported(const PrefillArgs& a, int total_tokens);
 int prefill_rows_per_entry(int n_q_heads, int n_kv_heads);   // query rows one plan entry covers: 128 or 256
 int prefill_plan_entries(const earn_batch_t& b, int rows);   // (sequence, block of `rows` query rows) pairs of the batch
+// One plan entry per (sequence, block of `rows` rows): {first global row, rows of the sequence from there, block index,
+// sequence}, blocks with the highest index (the longest key range) first; at most 2048 blocks per sequence.
+cudaError_t launch_tile_plan(const int32_t* cu_seqlens, int batch, int max_seqlen, int rows, void* plan, cudaStream_t st);
 // plan: device scratch of 16 bytes per plan entry, filled by a planning kernel launched ahead of the main one
 cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int plan_entries, void* plan, int32_t* status_word,
                               cudaStream_t st);

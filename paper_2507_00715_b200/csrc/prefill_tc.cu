@@ -28,10 +28,9 @@
 //
 // Every mbarrier wait is bounded; when one runs out the CTA raises its abort flag, writes
 // EARN_ERR_TIMEOUT to the status word, drains what it has in flight, frees its TMEM and returns.
-#include <cudaTypedefs.h>
-
 #include "earn_common.cuh"
 #include "sm100_ptx.cuh"
+#include "tc_maps.cuh"
 
 namespace earn {
 namespace {
@@ -571,31 +570,16 @@ __global__ void __launch_bounds__(PLAN_THREADS) prefill_plan_kernel(const int32_
 // ------------------------------------------------------------------------------------------------
 // host side: tensor maps over the packed [total, H, 128] bf16 tensors, box = 64 columns x 1 head x 128 tokens
 // ------------------------------------------------------------------------------------------------
-PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
-  static PFN_cuTensorMapEncodeTiled_v12000 fn = [] {
-    void* f = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      f = nullptr;
-    return reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(f);
-  }();
-  return fn;
-}
-
-bool make_map(CUtensorMap* map, const void* ptr, int heads, int total, int box_rows = BM) {
-  auto fn = encode_fn();
-  if (fn == nullptr) return false;
-  cuuint64_t dims[3] = {(cuuint64_t)HD, (cuuint64_t)heads, (cuuint64_t)total};
-  cuuint64_t strides[2] = {(cuuint64_t)HD * 2, (cuuint64_t)heads * HD * 2};
-  cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
-  cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
+using tcmap::make_map;
 
 }  // namespace
+
+cudaError_t launch_tile_plan(const int32_t* cu_seqlens, int batch, int max_seqlen, int rows, void* plan, cudaStream_t st) {
+  const cudaError_t e = launch_pdl(prefill_plan_kernel, dim3(1), dim3(PLAN_THREADS), 0, st, cu_seqlens, batch,
+                                   (max_seqlen + rows - 1) / rows, rows, reinterpret_cast<int4*>(plan));
+  note_launch();
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
 
 int prefill_rows_per_entry(int n_q_heads, int n_kv_heads) {
   // an even group: the two M-tiles of an item are two heads on the same 128 rows; otherwise two consecutive query tiles
@@ -615,15 +599,12 @@ bool prefill_tc_supported(const PrefillArgs& a, int total_tokens) {
 cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int plan_entries, void* plan, int32_t* status_word,
                               cudaStream_t st) {
   CUtensorMap mq, mk, mv, mo;
-  if (!make_map(&mq, a.q, a.Hq, total_tokens) || !make_map(&mk, a.k, a.Hkv, total_tokens) ||
-      !make_map(&mv, a.v, a.Hkv, total_tokens) || !make_map(&mo, a.o, a.Hq, total_tokens, 32))   // O leaves in slabs of 32 rows, one per warp
+  if (!make_map(&mq, a.q, a.Hq, total_tokens, BM) || !make_map(&mk, a.k, a.Hkv, total_tokens, BM) ||
+      !make_map(&mv, a.v, a.Hkv, total_tokens, BM) || !make_map(&mo, a.o, a.Hq, total_tokens, 32))   // O leaves in slabs of 32 rows, one per warp
     return cudaErrorInvalidValue;
   if (plan_entries <= 0) return cudaSuccess;
   const int rows = prefill_rows_per_entry(a.Hq, a.Hkv);
-  cudaError_t e = launch_pdl(prefill_plan_kernel, dim3(1), dim3(PLAN_THREADS), 0, st, a.cu_seqlens, a.batch,
-                             (a.max_seqlen + rows - 1) / rows, rows, reinterpret_cast<int4*>(plan));
-  note_launch();
-  if (e == cudaSuccess) e = cudaGetLastError();
+  cudaError_t e = launch_tile_plan(a.cu_seqlens, a.batch, a.max_seqlen, rows, plan, st);
   if (e != cudaSuccess) return e;
   TcParams p{};
   p.o = a.o; p.lse = a.lse; p.plan = reinterpret_cast<const int4*>(plan); p.status = status_word;

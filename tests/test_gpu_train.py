@@ -112,3 +112,24 @@ def test_full_layers_small_ragged(kw):
 def test_participating_layers(rh, rt, nt):
     run_participating_layer(SMALL.replace(r_head=rh, r_tail=rt), n_target=nt)
     run_participating_layer(SMALL.replace(r_head=rh, r_tail=rt, dtype="f32", head_dim=64, n_q_heads=4), n_target=nt)
+
+
+def test_full_layer_7b_shapes_sampled_sequences():
+    """The measured shape (64 sequences of 1024 tokens, 32 query heads over 8 kv heads): O, LSE, dQ, dK, dV of two whole
+    sequences (the first and the last) against the oracle; eight key tiles per sequence, groups of four heads adding
+    into each kv head, 36 (query tile, key tile) pairs per head."""
+    run_full_layer(wl.CONFIGS["7b"].replace(n_layers=2, split_k=1, decode_steps=0), sample_seqs=(0, 63))
+
+
+def test_full_layer_long_and_ragged_sampled_sequences():
+    w = wl.CONFIGS["ragged"].replace(n_layers=2, split_k=1, decode_steps=0, beams=1, batch=24)
+    lens = wl.seqlens(w)
+    run_full_layer(w, sample_seqs=(int(np.argmin(lens)), int(np.argmax(lens)), 23))
+
+
+def test_backward_is_reproducible():
+    w = SMALL.replace(seed=52)
+    a = run_full_layer(w)
+    b = run_full_layer(w)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
