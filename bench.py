@@ -123,6 +123,9 @@ def algorithmic(w: wl.Workload):
     qo = 2 * B * W * Hq * D * es + 4 * B * W * Hkv * D * es
     out["decode_compact"] = dict(flops=4.0 * D * Hq * B * W * (R + s), bytes=float(2 * B * (R + W * s) * Hkv * D * es + qo))
     out["decode_full"] = dict(flops=4.0 * D * Hq * W * (tot + B * s), bytes=float(2 * (tot + B * W * s) * Hkv * D * es + qo))
+    out["train_fwd"] = dict(flops=out["prefill"]["flops"], bytes=out["prefill"]["bytes"] + 4.0 * Hq * tot)
+    # backward: five products of the forward's two (S, dP, dV, dK, dQ); reads Q, K, V, O, dO, writes dQ, dK, dV
+    out["train_bwd"] = dict(flops=2.5 * out["prefill"]["flops"], bytes=float(tot * D * es * (4 * Hq + 4 * Hkv)))
     out["beam_topk"] = dict(flops=0.0, bytes=float(B * W * BEAM_VOCAB * 4 + B * W * 16))
     return out
 
@@ -324,6 +327,20 @@ class GpuJob:
                                                                               ses.x_norm, caches[l], self.q_reg, ses.workspace)
                                                      for i, l in enumerate(late)], len(late))
                 del x, wts
+        if early and w.dtype == "bf16":
+            # training-time attention of one full layer (Section 3.2 "Training"; not part of the timed inference step):
+            # forward with LSE, then backward (dQ, dK, dV); useful flops: forward 4 D per causal pair and head, backward 2.5 x
+            q, k, v = self.qkv[0]
+            total = q.shape[0]
+            tws = torch.empty(self.B.earn_train_workspace_bytes(ses.model, ses.batch), dtype=torch.uint8, device=self.dev)
+            self.B.earn_workspace_init(tws)
+            lse = torch.empty(w.n_q_heads, total, dtype=torch.float32, device=self.dev)
+            d_o = wl.upstream_grad(w, 0, q.shape, self.dev)
+            dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+            res["train_fwd"] = timed(lambda: self.B.earn_train_attn_fwd(ses.model, ses.batch, 0, 0, q, k, v, self.o_full, lse, tws), 1)
+            res["train_bwd"] = timed(lambda: self.B.earn_train_attn_bwd(ses.model, ses.batch, 0, 0, q, k, v, self.o_full, lse, d_o,
+                                                                        dq, dk, dv, tws), 1)
+            del tws, lse, d_o, dq, dk, dv
         if w.beams > 1:
             # beam selection between decode steps (not part of the timed step, which has no output layer to produce
             # log-probabilities): every log-probability read once, B * W * V * 4 bytes
