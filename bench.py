@@ -50,7 +50,7 @@ def read_peaks():
 
 
 KERNEL_SOURCES = {"prefill": "prefill_tc.cu", "compact": "compact.cu", "register": "register_mma.cu", "register_qkv": "register_qkv.cu",
-                  "decode_compact": "decode_mma.cu", "decode_full": "decode_mma.cu"}
+                  "register_layer": "register_mma.cu", "decode_compact": "decode_short.cu", "decode_full": "decode_mma.cu"}
 
 
 def source_digest(fname: str) -> str:
@@ -123,6 +123,7 @@ def algorithmic(w: wl.Workload):
     qo = 2 * B * W * Hq * D * es + 4 * B * W * Hkv * D * es
     out["decode_compact"] = dict(flops=4.0 * D * Hq * B * W * (R + s), bytes=float(2 * B * (R + W * s) * Hkv * D * es + qo))
     out["decode_full"] = dict(flops=4.0 * D * Hq * W * (tot + B * s), bytes=float(2 * (tot + B * W * s) * Hkv * D * es + qo))
+    out["compact_register"] = dict(flops=out["register"]["flops"], bytes=out["compact"]["bytes"] + out["register"]["bytes"])
     out["train_fwd"] = dict(flops=out["prefill"]["flops"], bytes=out["prefill"]["bytes"] + 4.0 * Hq * tot)
     # backward: five products of the forward's two (S, dP, dV, dK, dQ); reads Q, K, V, O, dO, writes dQ, dK, dV
     out["train_bwd"] = dict(flops=2.5 * out["prefill"]["flops"], bytes=float(tot * D * es * (4 * Hq + 4 * Hkv)))
@@ -205,6 +206,7 @@ class GpuJob:
         self.q_reg = torch.empty(w.batch, w.n_regs, w.n_q_heads, w.head_dim, **kw)
         self.o_reg = torch.empty_like(self.q_reg)
         self.o_dec = torch.empty(w.batch * w.beams, w.n_q_heads, w.head_dim, **kw)
+        self.fused_register = w.dtype == "bf16" and 0 < w.n_regs <= 128
         self.graphs = None
         self.marks = []
 
@@ -225,8 +227,14 @@ class GpuJob:
             segs.append(("prefill", len(early),
                          lambda: [ses.prefill_layer(l, *self.qkv[l], out=self.o_full) for l in early]))
         if late:
-            segs.append(("register_layer", len(late),
-                         lambda: [ses.prefill_layer(l, *self.qkv[l], out=self.o_reg, q_reg=self.q_reg) for l in late]))
+            # register layers: compaction + register attention, in one launch where the library has the fused kernel
+            # (bf16, at most 128 registers), through the two calls otherwise
+            if self.fused_register:
+                segs.append(("register_layer", len(late),
+                             lambda: [ses.register_layer_fused(l, *self.qkv[l], out=self.o_reg) for l in late]))
+            else:
+                segs.append(("register_layer", len(late),
+                             lambda: [ses.prefill_layer(l, *self.qkv[l], out=self.o_reg, q_reg=self.q_reg) for l in late]))
         for s in range(1, w.decode_steps + 1):
             if early:
                 def f(s=s):
@@ -316,6 +324,8 @@ class GpuJob:
                                                                    caches[l], self.qkv[l][0], self.q_reg) for l in late], len(late))
             res["register"] = timed(lambda: [self.B.earn_register_attn(ses.model, ses.batch, l, self.q_reg, caches[l],
                                                                        self.o_reg, ses.workspace) for l in late], len(late))
+            if self.fused_register:
+                res["compact_register"] = timed(lambda: [ses.register_layer_fused(l, *self.qkv[l], out=self.o_reg) for l in late], len(late))
             if w.dtype == "bf16" and w.head_dim == 128 and w.n_regs > 0:
                 # the same layers from hidden states (not part of the timed step, whose inputs are Q, K, V): one x for
                 # every layer, weights per layer so that they come from HBM as they would in a model
@@ -413,7 +423,10 @@ class GpuJob:
                 ses.prefill_layer(layer, q, k, v, out=out)
                 host = self.h_o_full[layer]
             else:
-                ses.prefill_layer(layer, q, k, v, out=out, q_reg=self.q_reg)
+                if self.fused_register:
+                    ses.register_layer_fused(layer, q, k, v, out=out)
+                else:
+                    ses.prefill_layer(layer, q, k, v, out=out, q_reg=self.q_reg)
                 host = self.h_o_reg[layer - w.split_k]
             done = torch.cuda.Event()
             done.record(cs)
@@ -525,6 +538,8 @@ def profile_one_kernel(w: wl.Workload, dev, which: str, launches: int = 3):
             B.earn_compact_kv(ses.model, ses.batch, 1, k, v, ses.cache(1), q, q_reg)
         elif which == "register":
             B.earn_register_attn(ses.model, ses.batch, 1, q_reg, ses.cache(1), o_reg, ses.workspace)
+        elif which == "register_layer":
+            ses.register_layer_fused(1, q, k, v, out=o_reg)
         elif which == "register_qkv":
             B.earn_register_qkv(ses.model, ses.batch, 1, proj, x, w_norm, w_qkv, ses.x_norm, ses.cache(1), q_reg, ses.workspace)
         else:
@@ -661,7 +676,7 @@ def parse_args(argv=None):
     ap.add_argument("--no-parts", action="store_true")
     ap.add_argument("--no-graphs", action="store_true", help="plain launches instead of CUDA-graph replay")
     ap.add_argument("--profile-kernel", default=None,
-                    choices=["prefill", "compact", "register", "register_qkv", "decode_compact", "decode_full"],
+                    choices=["prefill", "compact", "register", "register_layer", "register_qkv", "decode_compact", "decode_full"],
                     help="small case for a profiler: allocate ONE layer of the workload and launch that step 3 times")
     ap.add_argument("--sweep-k", default=None,
                     help="comma-separated split layers k: time the workload once per k (one JSON line each, k = N is the "
@@ -818,10 +833,7 @@ def main(argv=None, backend: str = "nccl", job_factory=None):
             ach = a["bytes"] / sec / 1e9
             r.update(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
                      frac_nominal=ach / NOMINAL["hbm_gbs"], peak_source=peaks["source"] + " (copy)")
-        if kind == "register_layer":
-            tr = traffic.get("compact", 0) + traffic.get("register", 0) if {"compact", "register"} <= set(traffic) else None
-        else:
-            tr = traffic.get(kind)
+        tr = traffic.get(kind)
         r.update(traffic=tr, avg_launch_ms=sec * 1e3, launches_per_step=per_step, share_of_step=share,
                  algorithmic_flops_per_launch=a["flops"], algorithmic_bytes_per_launch=a["bytes"])
         rooflines[kind] = r

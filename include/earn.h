@@ -174,6 +174,15 @@ earn_status_t earn_register_attn(const earn_model_t* model, const earn_batch_t* 
                                  const void* q_reg, const earn_cache_t* cache, void* o_reg,
                                  void* workspace, size_t workspace_bytes, earn_stream_t stream);
 
+/* Steps 2 and 3 in one launch (an additional call; the two above stay as they are): for a layer l >= k, read the register
+ * rows of q, k, v straight from the packed prompt tensors (Section 3.2, X -> X' = [prefix; suffix]), write the K and V rows
+ * into the compact cache pages and idx into cache->reg_idx exactly as earn_compact_kv does (bit copies), and compute the
+ * causal attention among the R register tokens as earn_register_attn does: o_reg, device [B, R, Hq, D].  No gathered copy
+ * of the queries is made.  bf16 with R <= 128 only; anything else -> EARN_ERR_UNSUPPORTED (use the two calls). */
+earn_status_t earn_compact_register_attn(const earn_model_t* model, const earn_batch_t* batch, int32_t layer,
+                                         const void* q, const void* k, const void* v, const earn_cache_t* cache,
+                                         void* o_reg, void* workspace, size_t workspace_bytes, earn_stream_t stream);
+
 /* Step 4 — one decode step of one layer (Eq. 4: append K_t, V_t, then attend over K_{1:t}, self included).
  * step is 1-based; beam j = b*W + w.  k_new/v_new (device [B*W, Hkv, D]) are stored at row (j, step-1) of the
  * private segment; q, o: device [B*W, Hq, D].  Keys seen by beam j:

@@ -62,6 +62,8 @@ SYMBOLS = {
                                     C.c_size_t, C.c_void_p]),
     "earn_register_attn": (C.c_int, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32, C.c_void_p,
                                      C.POINTER(EarnCache), C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "earn_compact_register_attn": (C.c_int, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32, C.c_void_p, C.c_void_p,
+                                             C.c_void_p, C.POINTER(EarnCache), C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "earn_decode_attn": (C.c_int, [C.POINTER(EarnModel), C.POINTER(EarnBatch), C.c_int32, C.c_int32, C.c_void_p,
                                    C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(EarnCache), C.c_void_p,
                                    C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -223,6 +225,12 @@ def earn_register_attn(model, batch: Batch, layer, q_reg, cache: EarnCache, o_re
     p, n = _ws(workspace)
     _check(lib().earn_register_attn(C.byref(model), C.byref(batch.c), layer, _ptr(q_reg), C.byref(cache), _ptr(o_reg),
                                     p, n, _stream()), "earn_register_attn")
+
+
+def earn_compact_register_attn(model, batch: Batch, layer, q, k, v, cache: EarnCache, o_reg, workspace=None) -> None:
+    p, n = _ws(workspace)
+    _check(lib().earn_compact_register_attn(C.byref(model), C.byref(batch.c), layer, _ptr(q), _ptr(k), _ptr(v),
+                                            C.byref(cache), _ptr(o_reg), p, n, _stream()), "earn_compact_register_attn")
 
 
 def earn_decode_attn(model, batch: Batch, layer, step, q, k_new, v_new, cache: EarnCache, o, k_full=None, v_full=None,

@@ -350,6 +350,33 @@ earn_status_t earn_register_attn(const earn_model_t* model, const earn_batch_t* 
   return e == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
 }
 
+earn_status_t earn_compact_register_attn(const earn_model_t* model, const earn_batch_t* batch, int32_t layer,
+                                         const void* q, const void* k, const void* v, const earn_cache_t* cache,
+                                         void* o_reg, void* workspace, size_t workspace_bytes, earn_stream_t stream) {
+  earn_status_t s = check_model(model);
+  if (s != EARN_OK) return s;
+  s = check_batch(batch);
+  if (s != EARN_OK) return s;
+  if (layer < model->split_k || layer >= model->n_layers) return EARN_ERR_INVALID_ARG;
+  s = check_cache_shared(model, batch, cache);
+  if (s != EARN_OK) return s;
+  const int R = batch->n_head_reg + batch->n_tail_reg;
+  if (R == 0 || batch->batch == 0) return EARN_OK;
+  if (!q || !k || !v || !o_reg || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o_reg)) return EARN_ERR_INVALID_ARG;
+  if (workspace == nullptr || workspace_bytes < (size_t)kStatusBytes) return EARN_ERR_WORKSPACE;
+  RegisterArgs a{};
+  a.q_reg = nullptr; a.o_reg = o_reg;
+  a.src = paged_source(batch, cache);
+  a.batch = batch->batch; a.R = R;
+  a.Hq = model->n_q_heads; a.Hkv = model->n_kv_heads; a.D = model->head_dim; a.dtype = model->dtype;
+  a.scale = scale_of(model);
+  a.q_full = q; a.k_full = k; a.v_full = v; a.cu_seqlens = batch->cu_seqlens; a.reg_idx = cache->reg_idx;
+  a.r_head = batch->n_head_reg; a.r_tail = batch->n_tail_reg;
+  if (!register_mma_supported(a)) return EARN_ERR_UNSUPPORTED;
+  note_call(stream, CALL_WRITES_CACHE);
+  return launch_register_mma(a, (cudaStream_t)stream) == cudaSuccess ? EARN_OK : EARN_ERR_CUDA;
+}
+
 earn_status_t earn_decode_attn(const earn_model_t* model, const earn_batch_t* batch, int32_t layer, int32_t step,
                                const void* q, const void* k_new, const void* v_new, const void* k_full_or_null,
                                const void* v_full_or_null, const earn_cache_t* cache, void* o, void* workspace,

@@ -129,6 +129,13 @@ struct RegisterArgs {
   KeySource src;
   int batch, R, Hq, Hkv, D, dtype;
   float scale;
+  // fused with the compaction (bf16 tensor-core kernel only): when k_full is not null the register rows of q, k, v are
+  // read straight from the packed prompt tensors (row cu_seqlens[b] + idx_b[m]); K and V are also written to the
+  // cache pages `src` names and idx to reg_idx, so that the call leaves what earn_compact_kv leaves
+  const void *q_full, *k_full, *v_full;
+  const int32_t* cu_seqlens;
+  int32_t* reg_idx;
+  int r_head, r_tail;
 };
 cudaError_t launch_register_simt(const RegisterArgs& a, cudaStream_t st);
 bool register_mma_supported(const RegisterArgs& a);                      // bf16 and R <= 128

@@ -96,6 +96,15 @@ class EarnSession:
         self.last_q_reg = q_reg
         return o
 
+    def register_layer_fused(self, layer: int, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
+                             out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Layer >= k in one launch: compaction and register attention together (no gathered copy of the queries).
+        Returns O' [B,R,Hq,D]; the compact cache and reg_idx are left as prefill_layer leaves them."""
+        o = out if out is not None else torch.empty(self.batch.batch, self.R, self.Hq, self.D, device=self.device,
+                                                    dtype=self.dtype)
+        B.earn_compact_register_attn(self.model, self.batch, layer, q, k, v, self.cache(layer), o, self.workspace)
+        return o
+
     def set_projection(self, d_model: int, max_pos: int, theta: float = 10000.0, rms_eps: float = 1e-6) -> None:
         """Rotary tables (angles pos * theta^(-2i/D), evaluated in double, stored fp32) and the scratch the
         hidden-state form of the register layers needs."""

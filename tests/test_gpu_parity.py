@@ -198,3 +198,31 @@ def test_private_segment_behind_a_page_table(shape):
           "short_list_head_dim_64": dict(head_dim=64, n_q_heads=4, n_kv_heads=2, beams=2)}[shape]
     w = BASE.replace(seed=23, lens=(90, 40), batch=2, n_layers=2, split_k=1, r_head=4, r_tail=4, decode_steps=18, **kw)
     run_workload_and_compare(w, check_lse=False, paged_private_seed=9, paged_shuffle_seed=3)
+
+
+@pytest.mark.parametrize("kw", [dict(), dict(r_head=16, r_tail=16, paged=True), dict(n_q_heads=6, n_kv_heads=2, r_head=3, r_tail=4),
+                                dict(r_head=0, r_tail=4), dict(r_head=40, r_tail=37, n_q_heads=2, n_kv_heads=2, lens=(100, 300), batch=2),
+                                dict(r_head=3, r_tail=4, lens=(7, 8, 300)), dict(head_dim=64)])
+def test_compaction_and_register_attention_in_one_launch(kw):
+    """earn_compact_register_attn leaves the cache pages and the index list bit-identical to earn_compact_kv's and returns
+    earn_register_attn's output (here: bit-identical too, the arithmetic is the same kernel's), and both match the oracle."""
+    from parity_util import assert_close, make_session, to_np
+    from oracle import earn_oracle as orc
+    kw = dict(kw)
+    paged = kw.pop("paged", False)
+    w = BASE.replace(seed=24, n_layers=2, split_k=1, decode_steps=0, **kw)
+    cu = wl.cu_seqlens(w)
+    idx = orc.register_indices(wl.seqlens(w), w.r_head, w.r_tail)
+    q, k, v = wl.layer_qkv(w, 1, "cuda")
+    two = make_session(w, paged_shuffle_seed=5 if paged else None)
+    o_two = two.prefill_layer(1, q, k, v)
+    one = make_session(w, paged_shuffle_seed=5 if paged else None)
+    o_one = one.register_layer_fused(1, q, k, v)
+    torch.cuda.synchronize()
+    assert torch.equal(one.k_shared[1], two.k_shared[1]) and torch.equal(one.v_shared[1], two.v_shared[1])
+    assert torch.equal(one.reg_idx, two.reg_idx)
+    assert torch.equal(o_one, o_two)
+    qn, kn, vn = to_np(q), to_np(k), to_np(v)
+    assert_close(o_one, orc.register_attention(orc.compact(qn, cu, idx), orc.compact(kn, cu, idx), orc.compact(vn, cu, idx)),
+                 w.dtype, "fused register layer")
+    assert np.array_equal(one.reg_idx.cpu().numpy()[:, :w.n_regs], idx)
