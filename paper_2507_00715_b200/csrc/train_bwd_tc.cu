@@ -19,9 +19,10 @@
 // so every tensor-core product has the shapes and operand layouts of the forward kernel's two (left operand K-major
 // from shared memory, or from tensor memory; right operand K-major or MN-major from a TMA-loaded tile).
 //   warp 0  TMA producer    warp 1  tcgen05.mma issuer (and TMEM owner)    warps 4-7  the softmax warpgroup
-// The next X, Y of an item are issued behind the accumulating products of the tile before (which read p and ds from the
-// columns X and Y are written to); all 512 TMEM columns are taken (X, Y, acc0, acc1), so there is no second X / Y to
-// work ahead on, and the tensor core and the softmax warpgroup take turns within an item.
+// All 512 TMEM columns are taken (X, Y, acc0, acc1), so there is no second X / Y to work ahead on; the overlap comes from
+// the issue order X(u) | acc1(u-1) | Y(u) | acc0(u): the warpgroup turns X into p while the tensor core does acc1 and Y,
+// and Y into ds while it does acc0 (issued tile by tile as X Y, then acc0 acc1, the tensor core and the warpgroup took
+// turns: 3.5 ms against the figures in the design doc for the 7B-class layer).
 // Every mbarrier wait is bounded as in the forward kernel.
 #include "earn_common.cuh"
 #include "sm100_ptx.cuh"
@@ -45,9 +46,9 @@ struct BCfg {
   static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;           // + alignment slack
   static constexpr int TMEM_COLS = 512;                             // X 0, Y 128, acc0 256, acc1 384
   static constexpr int THREADS = 256;
-  static constexpr int BAR_RES = 0, BAR_FULL = 1, BAR_EMPTY = BAR_FULL + NSTAGE, BAR_XY = BAR_EMPTY + NSTAGE,
-                       BAR_P = BAR_XY + 1, BAR_DS = BAR_P + 1, BAR_ACC = BAR_DS + 1, BAR_DRAIN = BAR_ACC + 1,
-                       N_BARS = BAR_DRAIN + 1;
+  static constexpr int BAR_RES = 0, BAR_FULL = 1, BAR_EMPTY = BAR_FULL + NSTAGE, BAR_X = BAR_EMPTY + NSTAGE,
+                       BAR_Y = BAR_X + 1, BAR_P = BAR_Y + 1, BAR_DS = BAR_P + 1, BAR_ACC = BAR_DS + 1,
+                       BAR_DRAIN = BAR_ACC + 1, N_BARS = BAR_DRAIN + 1;
 };
 
 struct BwdParams {
@@ -122,7 +123,8 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       mbar_init(bar(C::BAR_FULL + s), 1);
       mbar_init(bar(C::BAR_EMPTY + s), 1);
     }
-    mbar_init(bar(C::BAR_XY), 1);
+    mbar_init(bar(C::BAR_X), 1);
+    mbar_init(bar(C::BAR_Y), 1);
     mbar_init(bar(C::BAR_P), 128);
     mbar_init(bar(C::BAR_DS), 128);
     mbar_init(bar(C::BAR_ACC), 1);
@@ -210,18 +212,22 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           umma_ts_lohi(d_tmem, a_tmem + kk * 8, b_lo + kk * (2048 >> 4), desc_hi, idesc_acc, (!first || kk > 0) ? 1u : 0u);
       }
     };
-    bool ok = wait(C::BAR_RES, 0);
-    for (int u = 0; u < job.n_iter && ok; ++u) {
-      const int st = u % C::NSTAGE;
-      const uint32_t t0 = sT + st * 2 * TILE, t1 = t0 + TILE;
-      ok = wait(C::BAR_FULL + st, u / C::NSTAGE);
-      if (!ok) break;
+    // Order on the tensor core, per streamed tile u:  X(u) | acc1(u-1) | Y(u) | acc0(u)  -- the softmax warpgroup turns
+    // X(u) into p while acc1(u-1) and Y(u) run, and Y(u) into ds while acc0(u) runs.  One thread's tensor-core instructions
+    // run in the order they were issued, which is what lets X(u) go over the columns acc0(u-1) read p from, and Y(u)
+    // over the columns acc1(u-1) reads ds from.
+    bool ok = wait(C::BAR_RES, 0) && wait(C::BAR_FULL + 0, 0);
+    if (ok) {
       tc_fence_after();
-      // (issued behind the accumulating products of tile u - 1, which read p and ds out of these columns: one thread's
-      // tensor-core instructions run in the order they were issued)
-      issue_xy(tmem + 0, l_lo, smem_desc_lo(t0, 16));
-      issue_xy(tmem + 128, l_lo + (TILE >> 4), smem_desc_lo(t1, 16));
-      if (leader) umma_commit(bar(C::BAR_XY));
+      issue_xy(tmem + 0, l_lo, smem_desc_lo(sT, 16));
+      if (leader) umma_commit(bar(C::BAR_X));
+      issue_xy(tmem + 128, l_lo + (TILE >> 4), smem_desc_lo(sT + TILE, 16));
+      if (leader) umma_commit(bar(C::BAR_Y));
+    }
+    for (int u = 0; u < job.n_iter && ok; ++u) {
+      const int st = u % C::NSTAGE, sn = (u + 1) % C::NSTAGE;
+      const uint32_t t0 = sT + st * 2 * TILE, t1 = t0 + TILE, n0 = sT + sn * 2 * TILE, n1 = n0 + TILE;
+      const bool more = u + 1 < job.n_iter;
       if (MODE == MODE_KV) {
         ok = wait(C::BAR_P, u);
         if (!ok) break;
@@ -229,12 +235,21 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         issue_acc(tmem + 256, tmem + 0, t1, u == 0);      // dV += P^T dO
       }
       ok = wait(C::BAR_DS, u);
+      if (ok && more) ok = wait(C::BAR_FULL + sn, (u + 1) / C::NSTAGE);
       if (!ok) break;
       tc_fence_after();
+      if (more) {
+        issue_xy(tmem + 0, l_lo, smem_desc_lo(n0, 16));
+        if (leader) umma_commit(bar(C::BAR_X));
+      }
       issue_acc(tmem + 384, tmem + 128, t0, u == 0);      // dK += dS^T Q   or   dQ += dS K
       if (leader) {
         umma_commit(bar(C::BAR_EMPTY + st));
-        if (u == job.n_iter - 1) umma_commit(bar(C::BAR_ACC));
+        if (!more) umma_commit(bar(C::BAR_ACC));
+      }
+      if (more) {
+        issue_xy(tmem + 128, l_lo + (TILE >> 4), smem_desc_lo(n1, 16));
+        if (leader) umma_commit(bar(C::BAR_Y));
       }
     }
     if (leader && *abort_flag) {
@@ -286,7 +301,7 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         asm volatile("bar.sync 1, 128;" ::: "memory");   // the warpgroup's own barrier
         fetch_stat(u + 1, nx_lse, nx_delta);
       }
-      ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_XY), u & 1, abort_flag, WAIT_LIMIT));
+      ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_X), u & 1, abort_flag, WAIT_LIMIT));
       if (!ok) break;
       tc_fence_after();
       // column c of the tile pairs with this lane iff both belong to the sequence and the key is not after the query:
@@ -323,6 +338,9 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         mbar_arrive(bar(C::BAR_P));
       }
       // ---- pass 2: ds = p (y - delta) as bf16 pairs, written over the columns of y already read
+      ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_Y), u & 1, abort_flag, WAIT_LIMIT));
+      if (!ok) break;
+      tc_fence_after();
       tmem_ld_32x32(t_y, a);
       tmem_wait_ld(a);
 #pragma unroll
