@@ -18,7 +18,7 @@
 //   MODE_KV: acc0 += p T1 (dV += P^T dO)      both modes: acc1 += ds T0 (dK += dS^T Q  or  dQ += dS K)
 // so every tensor-core product has the shapes and operand layouts of the forward kernel's two (left operand K-major
 // from shared memory, or from tensor memory; right operand K-major or MN-major from a TMA-loaded tile).
-//   warp 0  TMA producer    warp 1  tcgen05.mma issuer (and TMEM owner)    warps 4-7  the softmax warpgroup
+//   warp 0  TMA producer    warp 1  tcgen05.mma issuer (and TMEM owner)    warps 4-11  two softmax warpgroups, 64 columns each
 // All 512 TMEM columns are taken (X, Y, acc0, acc1), so there is no second X / Y to work ahead on; the overlap comes from
 // the issue order X(u) | acc1(u-1) | Y(u) | acc0(u): the warpgroup turns X into p while the tensor core does acc1 and Y,
 // and Y into ds while it does acc0 (issued tile by tile as X Y, then acc0 acc1, the tensor core and the warpgroup took
@@ -45,7 +45,7 @@ struct BCfg {
   static constexpr int OFF_BAR = OFF_STAT + NSTAGE * 2 * BM * 4;
   static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;           // + alignment slack
   static constexpr int TMEM_COLS = 512;                             // X 0, Y 128, acc0 256, acc1 384
-  static constexpr int THREADS = 256;
+  static constexpr int THREADS = 384;                               // TMA, MMA, two idle warps, two softmax warpgroups
   static constexpr int BAR_RES = 0, BAR_FULL = 1, BAR_EMPTY = BAR_FULL + NSTAGE, BAR_X = BAR_EMPTY + NSTAGE,
                        BAR_Y = BAR_X + 1, BAR_P = BAR_Y + 1, BAR_DS = BAR_P + 1, BAR_ACC = BAR_DS + 1,
                        BAR_DRAIN = BAR_ACC + 1, N_BARS = BAR_DRAIN + 1;
@@ -125,8 +125,8 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     }
     mbar_init(bar(C::BAR_X), 1);
     mbar_init(bar(C::BAR_Y), 1);
-    mbar_init(bar(C::BAR_P), 128);
-    mbar_init(bar(C::BAR_DS), 128);
+    mbar_init(bar(C::BAR_P), 256);
+    mbar_init(bar(C::BAR_DS), 256);
     mbar_init(bar(C::BAR_ACC), 1);
     mbar_init(bar(C::BAR_DRAIN), 1);
     *abort_flag = 0;
@@ -259,9 +259,12 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     }
     __syncwarp();
   } else if (warp >= 4) {
-    // ------------------------------------------------------------------ softmax warpgroup: thread = lane l of tensor memory
-    const int wq = warp & 3, l = wq * 32 + lane;
-    const uint32_t t_x = tmem + ((uint32_t)(wq * 32) << 16), t_y = t_x + 128;
+    // ------------------------------------------------------------------ two softmax warpgroups: thread = lane l of tensor
+    // memory; warpgroup wg takes columns 64 wg .. 64 wg + 63 of X and of Y (one warpgroup over all 128 columns was bound
+    // by the instructions one warp per scheduler can issue: about 1900 clocks per pass)
+    const int wq = warp & 3, l = wq * 32 + lane, wg = (warp - 4) >> 2, c0 = wg * 64;
+    const uint32_t t_lane = tmem + ((uint32_t)(wq * 32) << 16);
+    const uint32_t t_x = t_lane + c0, t_y = t_lane + 128 + c0;
     const float sl2 = p.scale_log2;
     // MODE_Q: the thread's own query row has one LSE and one delta for the whole item
     float my_lse = 0.f, my_delta = 0.f;
@@ -270,12 +273,12 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       my_lse = __ldg(p.lse2 + at);
       my_delta = __ldg(p.delta + at);
     }
-    // MODE_KV: LSE and delta belong to the streamed query rows: thread l fetches those of row l of the tile one
-    // iteration ahead and the warpgroup shares them through shared memory
+    // MODE_KV: LSE and delta belong to the streamed query rows: thread l of the first warpgroup fetches those of row l
+    // of the tile one iteration ahead and both warpgroups read them from shared memory
     auto fetch_stat = [&](int u, float& a_lse, float& a_delta) {
       a_lse = 0.f;
       a_delta = 0.f;
-      if (MODE == MODE_KV && u < job.n_iter) {
+      if (MODE == MODE_KV && wg == 0 && u < job.n_iter) {
         const int it = u % job.n_t;
         if (it * BM + l < job.rows_left) {
           const int64_t at = (int64_t)t_head(u) * p.total + t_row(u) + l;
@@ -289,16 +292,19 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     bool ok = true;
     for (int u = 0; u < job.n_iter && ok; ++u) {
       const int st = u % C::NSTAGE;
-      float* s_lse = stat + st * 2 * BM;
-      float* s_delta = s_lse + BM;
+      const float* s_lse = stat + st * 2 * BM;
+      const float* s_delta = s_lse + BM;
       // streamed tile index within the sequence relative to the left tile (0 = the diagonal tile), valid columns
       const int rel = MODE == MODE_KV ? u % job.n_t : job.n_t - 1 - u;
       const bool diag = rel == 0;
       const int col_valid = MODE == MODE_KV ? min(job.rows_left - rel * BM, BM) : BM;   // MODE_KV: query rows of the sequence in this tile
+      const bool masked = diag || col_valid < BM;   // warp-uniform: interior tiles take the path without compares
       if (MODE == MODE_KV) {
-        s_lse[l] = nx_lse;
-        s_delta[l] = nx_delta;
-        asm volatile("bar.sync 1, 128;" ::: "memory");   // the warpgroup's own barrier
+        if (wg == 0) {
+          stat[st * 2 * BM + l] = nx_lse;
+          stat[st * 2 * BM + BM + l] = nx_delta;
+        }
+        asm volatile("bar.sync 1, 256;" ::: "memory");   // the softmax warps' own barrier
         fetch_stat(u + 1, nx_lse, nx_delta);
       }
       ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_X), u & 1, abort_flag, WAIT_LIMIT));
@@ -307,75 +313,88 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       // column c of the tile pairs with this lane iff both belong to the sequence and the key is not after the query:
       //   MODE_KV: lane = key, column = query row: c >= l on the diagonal tile, c < col_valid always
       //   MODE_Q : lane = query row, column = key: c <= l on the diagonal tile (keys past the sequence lie past every valid row)
-      uint32_t a[32], b[32], pk[4][16];
-      // ---- pass 1: p = 2^(x c log2e - LSE) as bf16 pairs
+      uint32_t a[32], b[32], pk[2][16];
+      // ---- p = 2^(x c log2e - LSE) as bf16 pairs.  p goes over the first 64 columns of X, so the second warpgroup's
+      // share lands on columns the first one reads: everybody has X in registers before anybody writes.
       tmem_ld_32x32(t_x, a);
+      tmem_ld_32x32(t_x + 32, b);
       tmem_wait_ld(a);
+      tmem_wait_ld(b);
+      if (MODE == MODE_KV) asm volatile("bar.sync 2, 256;" ::: "memory");
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint32_t(&cur)[32] = (q & 1) ? b : a;
-        uint32_t(&nxt)[32] = (q & 1) ? a : b;
-        if (q + 1 < 4) tmem_ld_32x32(t_x + (q + 1) * 32, nxt);
+      for (int q = 0; q < 2; ++q) {
+        uint32_t(&cur)[32] = q ? b : a;
 #pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          float e[2];
+        for (int c = 0; c < 32; c += 4) {
+          const int col = c0 + q * 32 + c;
+          float4 ls = make_float4(my_lse, my_lse, my_lse, my_lse);
+          if (MODE == MODE_KV) ls = *reinterpret_cast<const float4*>(s_lse + col);
+          float e[4];
+          e[0] = ex2(fmaf(__uint_as_float(cur[c + 0]), sl2, -ls.x));
+          e[1] = ex2(fmaf(__uint_as_float(cur[c + 1]), sl2, -ls.y));
+          e[2] = ex2(fmaf(__uint_as_float(cur[c + 2]), sl2, -ls.z));
+          e[3] = ex2(fmaf(__uint_as_float(cur[c + 3]), sl2, -ls.w));
+          if (masked) {
 #pragma unroll
-          for (int z = 0; z < 2; ++z) {
-            const int col = q * 32 + c + z;
-            const float lse = MODE == MODE_KV ? s_lse[col] : my_lse;
-            const bool seen = MODE == MODE_KV ? (col < col_valid && (!diag || col >= l)) : (!diag || col <= l);
-            e[z] = seen ? ex2(fmaf(__uint_as_float(cur[c + z]), sl2, -lse)) : 0.f;
+            for (int z = 0; z < 4; ++z) {
+              const bool seen = MODE == MODE_KV ? (col + z < col_valid && (!diag || col + z >= l)) : (!diag || col + z <= l);
+              if (!seen) e[z] = 0.f;
+            }
           }
           pk[q][c >> 1] = pack_bf16(e[0], e[1]);
+          pk[q][(c >> 1) + 1] = pack_bf16(e[2], e[3]);
         }
-        if (q + 1 < 4) tmem_wait_ld(nxt);
       }
+      ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_Y), u & 1, abort_flag, WAIT_LIMIT));
+      if (!ok) break;
+      tc_fence_after();
+      tmem_ld_32x32(t_y, a);        // Y on its way while p is stored
+      tmem_ld_32x32(t_y + 32, b);
       if (MODE == MODE_KV) {
-#pragma unroll
-        for (int q = 0; q < 4; ++q) tmem_st_32x16(t_x + q * 16, pk[q]);
+        tmem_st_32x16(t_lane + wg * 32, pk[0]);
+        tmem_st_32x16(t_lane + wg * 32 + 16, pk[1]);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(bar(C::BAR_P));
       }
-      // ---- pass 2: ds = p (y - delta) as bf16 pairs, written over the columns of y already read
-      ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_Y), u & 1, abort_flag, WAIT_LIMIT));
-      if (!ok) break;
-      tc_fence_after();
-      tmem_ld_32x32(t_y, a);
       tmem_wait_ld(a);
+      tmem_wait_ld(b);
+      asm volatile("bar.sync 3, 256;" ::: "memory");   // everybody has Y in registers before ds goes over its first 64 columns
+      // ---- ds = p (y - delta) as bf16 pairs (p is exactly zero where the pair is masked; the difference is finite there:
+      // every operand is real data or zero fill)
+      uint32_t dsk[2][16];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint32_t(&cur)[32] = (q & 1) ? b : a;
-        uint32_t(&nxt)[32] = (q & 1) ? a : b;
-        if (q + 1 < 4) tmem_ld_32x32(t_y + (q + 1) * 32, nxt);
-        uint32_t dsk[16];
+      for (int q = 0; q < 2; ++q) {
+        uint32_t(&cur)[32] = q ? b : a;
 #pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          const uint32_t pw = pk[q][c >> 1];
-          const float p0 = __uint_as_float(pw << 16), p1 = __uint_as_float(pw & 0xffff0000u);
-          const int col = q * 32 + c;
-          const float d0 = MODE == MODE_KV ? s_delta[col] : my_delta, d1 = MODE == MODE_KV ? s_delta[col + 1] : my_delta;
-          // (p is exactly zero where the pair is masked; the difference is finite there: every operand is real data or zero fill)
-          dsk[c >> 1] = pack_bf16(p0 * (__uint_as_float(cur[c]) - d0), p1 * (__uint_as_float(cur[c + 1]) - d1));
+        for (int c = 0; c < 32; c += 4) {
+          const int col = c0 + q * 32 + c;
+          float4 dl = make_float4(my_delta, my_delta, my_delta, my_delta);
+          if (MODE == MODE_KV) dl = *reinterpret_cast<const float4*>(s_delta + col);
+          const uint32_t pw0 = pk[q][c >> 1], pw1 = pk[q][(c >> 1) + 1];
+          dsk[q][c >> 1] = pack_bf16(__uint_as_float(pw0 << 16) * (__uint_as_float(cur[c + 0]) - dl.x),
+                                     __uint_as_float(pw0 & 0xffff0000u) * (__uint_as_float(cur[c + 1]) - dl.y));
+          dsk[q][(c >> 1) + 1] = pack_bf16(__uint_as_float(pw1 << 16) * (__uint_as_float(cur[c + 2]) - dl.z),
+                                           __uint_as_float(pw1 & 0xffff0000u) * (__uint_as_float(cur[c + 3]) - dl.w));
         }
-        if (q + 1 < 4) tmem_wait_ld(nxt);   // chunk q + 1 of y is in registers before ds overwrites any of it
-        tmem_st_32x16(t_y + q * 16, dsk);
       }
+      tmem_st_32x16(t_lane + 128 + wg * 32, dsk[0]);
+      tmem_st_32x16(t_lane + 128 + wg * 32 + 16, dsk[1]);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(bar(C::BAR_DS));
     }
-    // ---- the item's accumulators -> global memory
+    // ---- the item's accumulators -> global memory (each warpgroup its half of the columns)
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(bar(C::BAR_ACC), 0, abort_flag, WAIT_LIMIT));
     if (ok) {
       tc_fence_after();
       const bool valid = l < job.left_valid;
       uint32_t a[32];
       auto store_rows = [&](uint32_t t_acc, void* out, int heads, int head, float mul) {
-        __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(out) + ((int64_t)(job.left_row0 + l) * heads + head) * HD;
+        __nv_bfloat16* orow = reinterpret_cast<__nv_bfloat16*>(out) + ((int64_t)(job.left_row0 + l) * heads + head) * HD + c0;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          tmem_ld_32x32(t_acc + q * 32, a);
+        for (int q = 0; q < 2; ++q) {
+          tmem_ld_32x32(t_acc + c0 + q * 32, a);
           tmem_wait_ld(a);
           if (valid) {
 #pragma unroll
@@ -391,10 +410,10 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
       };
       if (MODE == MODE_KV) {
-        store_rows(t_x + 256, p.dv, p.Hkv, job.kvh, 1.f);
-        store_rows(t_x + 384, p.dk, p.Hkv, job.kvh, p.scale);
+        store_rows(t_lane + 256, p.dv, p.Hkv, job.kvh, 1.f);
+        store_rows(t_lane + 384, p.dk, p.Hkv, job.kvh, p.scale);
       } else {
-        store_rows(t_x + 384, p.dq, p.Hq, job.head0, p.scale);
+        store_rows(t_lane + 384, p.dq, p.Hq, job.head0, p.scale);
       }
     }
   }
