@@ -505,7 +505,7 @@ class OracleSample:
 
 def profile_one_kernel(w: wl.Workload, dev, which: str, launches: int = 3):
     """One layer of the workload, one kind of launch, `launches` times (a few GB at most on the device)."""
-    early = which in ("prefill", "decode_full")
+    early = which in ("prefill", "decode_full", "train_bwd")
     # keep the layer on the side of the split the kernel belongs to; one full layer + one register layer
     w1 = w.replace(n_layers=2, split_k=1)
     layer = 0 if early else 1
@@ -530,9 +530,26 @@ def profile_one_kernel(w: wl.Workload, dev, which: str, launches: int = 3):
         x = wl.hidden_states(w1, 1, dev)
         w_norm, w_qkv = wl.projection_weights(w1, 1, dev)
         proj = B.make_proj(w1.d_model, ses.rope_cos, ses.rope_sin)
+    if which == "train_bwd":
+        tws = torch.empty(B.earn_train_workspace_bytes(ses.model, ses.batch), dtype=torch.uint8, device=dev)
+        B.earn_workspace_init(tws)
+        lse = torch.empty(w1.n_q_heads, q.shape[0], dtype=torch.float32, device=dev)
+        d_o = wl.upstream_grad(w1, 0, q.shape, dev)
+        g_q, g_k, g_v = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+        B.earn_train_attn_fwd(ses.model, ses.batch, 0, 0, q, k, v, o, lse, tws)
+    if which == "beam_topk":
+        rows = w1.batch * w1.beams
+        lp = wl.beam_logprobs(w1, 1, BEAM_VOCAB, dev)
+        sc = [torch.zeros(rows, device=dev), torch.zeros(rows, device=dev)]
+        par, tok = (torch.zeros(rows, dtype=torch.int32, device=dev) for _ in range(2))
+        bws = torch.empty(B.earn_beam_topk_workspace_bytes(w1.batch, w1.beams, BEAM_VOCAB), dtype=torch.uint8, device=dev)
     torch.cuda.synchronize()
     for _ in range(launches):
-        if which == "prefill":
+        if which == "train_bwd":
+            B.earn_train_attn_bwd(ses.model, ses.batch, 0, 0, q, k, v, o, lse, d_o, g_q, g_k, g_v, tws)
+        elif which == "beam_topk":
+            B.earn_beam_topk(w1.batch, w1.beams, w1.beams, BEAM_VOCAB, lp, sc[0], par, tok, sc[1], bws)
+        elif which == "prefill":
             ses.prefill_layer(0, q, k, v, out=o)
         elif which == "compact":
             B.earn_compact_kv(ses.model, ses.batch, 1, k, v, ses.cache(1), q, q_reg)
@@ -676,7 +693,8 @@ def parse_args(argv=None):
     ap.add_argument("--no-parts", action="store_true")
     ap.add_argument("--no-graphs", action="store_true", help="plain launches instead of CUDA-graph replay")
     ap.add_argument("--profile-kernel", default=None,
-                    choices=["prefill", "compact", "register", "register_layer", "register_qkv", "decode_compact", "decode_full"],
+                    choices=["prefill", "compact", "register", "register_layer", "register_qkv", "decode_compact", "decode_full",
+                             "train_bwd", "beam_topk"],
                     help="small case for a profiler: allocate ONE layer of the workload and launch that step 3 times")
     ap.add_argument("--sweep-k", default=None,
                     help="comma-separated split layers k: time the workload once per k (one JSON line each, k = N is the "
