@@ -76,8 +76,12 @@ struct Job {
 template <int MODE>
 __device__ __forceinline__ Job make_job(const BwdParams& p) {
   Job j;
+  // The plan is sequence-major (all tiles of sequence 0, then of sequence 1, ...), low tile indices first: the CTAs that
+  // run at the same time then work on two or three sequences, whose Q / dO (MODE_KV) or K / V (MODE_Q) tiles they share
+  // through L2.  (Ordered by tile index over the whole batch, longest items first, the dK / dV launch read 5.2 GB from
+  // DRAM for a 7B-class layer whose Q and dO are 1.07 GB: every key tile's CTA fetched its query tiles afresh.)
   if (MODE == MODE_KV) {
-    const int e = p.n_entries - 1 - (int)blockIdx.x / p.Hkv;   // the plan lists high tile indices first; here low ones are the long items
+    const int e = (int)blockIdx.x / p.Hkv;
     const int4 t = __ldg(p.plan + e);
     j.kvh = blockIdx.x % p.Hkv;
     j.head0 = j.kvh * p.g;
@@ -88,16 +92,18 @@ __device__ __forceinline__ Job make_job(const BwdParams& p) {
     j.t_row0 = t.x;
     j.rows_left = t.y;
   } else {
+    // entry (sequence, tile z) stands for query tile nt - 1 - z here: within a sequence the long items come first
     const int e = (int)blockIdx.x / p.Hq;
     const int4 t = __ldg(p.plan + e);
+    const int lo = t.x - t.z * BM, len = t.y + t.z * BM, i = (len + BM - 1) / BM - 1 - t.z;
     j.head0 = blockIdx.x % p.Hq;
     j.kvh = j.head0 / p.g;
-    j.left_row0 = t.x;
-    j.left_valid = min(t.y, BM);
-    j.n_t = t.z + 1;
+    j.left_row0 = lo + i * BM;
+    j.left_valid = min(len - i * BM, BM);
+    j.n_t = i + 1;
     j.n_iter = j.n_t;
-    j.t_row0 = t.x - t.z * BM;
-    j.rows_left = t.y + t.z * BM;
+    j.t_row0 = lo;
+    j.rows_left = len;
   }
   return j;
 }
@@ -427,6 +433,35 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
   }
 }
 
+// Sequence-major plan: entry (sequence b, tile z) = {first global row of the tile, rows of the sequence from there, z, b}
+// at index (tiles of the sequences before b) + z.  One CTA; the sequences are scanned 1024 at a time.
+__global__ void __launch_bounds__(1024) train_plan_kernel(const int32_t* cu_seqlens, int batch, int4* plan) {
+  __shared__ int scan[1024];
+  __shared__ int carry;
+  pdl_launch_dependents();
+  pdl_wait();   // the plan area may still be read by the kernel before this one
+  if (threadIdx.x == 0) carry = 0;
+  __syncthreads();
+  for (int b0 = 0; b0 < batch; b0 += 1024) {
+    const int b = b0 + threadIdx.x;
+    const int lo = b < batch ? cu_seqlens[b] : 0, len = b < batch ? cu_seqlens[b + 1] - lo : 0;
+    const int nt = (len + BM - 1) / BM;
+    scan[threadIdx.x] = nt;
+    __syncthreads();
+    for (int off = 1; off < 1024; off <<= 1) {   // inclusive scan
+      const int add = threadIdx.x >= off ? scan[threadIdx.x - off] : 0;
+      __syncthreads();
+      scan[threadIdx.x] += add;
+      __syncthreads();
+    }
+    const int first = carry + scan[threadIdx.x] - nt;
+    for (int z = 0; z < nt; ++z) plan[first + z] = make_int4(lo + z * BM, len - z * BM, z, b);
+    __syncthreads();
+    if (threadIdx.x == 1023) carry += scan[1023];
+    __syncthreads();
+  }
+}
+
 // delta[h][row] = sum_d dO[row, h, d] * O[row, h, d] and the forward's LSE moved into the log2 domain: one warp per (row, head)
 __global__ void __launch_bounds__(256) train_bwd_prep_kernel(const __nv_bfloat16* o, const __nv_bfloat16* d_o, const float* lse,
                                                              float* delta, float* lse2, int total, int Hq) {
@@ -464,7 +499,9 @@ cudaError_t launch_train_bwd_tc(const TrainArgs& a, const earn_batch_t& b, void*
     return cudaErrorInvalidValue;
   const int n_entries = prefill_plan_entries(b, BM);
   if (n_entries <= 0) return cudaSuccess;
-  cudaError_t e = launch_tile_plan(a.cu_seqlens, a.batch, a.max_seqlen, BM, plan, st);
+  cudaError_t e = launch_pdl(train_plan_kernel, dim3(1), dim3(1024), 0, st, a.cu_seqlens, a.batch, reinterpret_cast<int4*>(plan));
+  note_launch();
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const int64_t warps = (int64_t)a.total * a.Hq;
   e = launch_pdl(train_bwd_prep_kernel, dim3((unsigned)((warps + 7) / 8)), dim3(256), 0, st,
