@@ -27,6 +27,7 @@ from paper_2507_00715_b200 import replicas, workloads as wl  # noqa: E402
 
 METRIC = "EARN attn tokens/s/GPU (prefill+decode, 7B GQA)"
 BEAM_VOCAB = 32000   # vocabulary the beam-selection kernel is timed on (the size of the paper's multi-head backbone's)
+L2_BYTES = 126 << 20   # B200
 UNIT = "tokens/s"
 
 
@@ -355,13 +356,16 @@ class GpuJob:
             # beam selection between decode steps (not part of the timed step, which has no output layer to produce
             # log-probabilities): every log-probability read once, B * W * V * 4 bytes
             vocab = BEAM_VOCAB
-            lp = wl.beam_logprobs(w, 1, vocab, self.dev)
             rows = w.batch * w.beams
+            # several inputs in turn, together larger than L2 (one of them may fit in it)
+            n_in = max(2, min(8, -(-(3 * L2_BYTES) // (rows * vocab * 4))))
+            lps = [wl.beam_logprobs(w, 1 + i, vocab, self.dev) for i in range(n_in)]
             sc = [torch.zeros(rows, device=self.dev), torch.zeros(rows, device=self.dev)]
             par, tok = (torch.zeros(rows, dtype=torch.int32, device=self.dev) for _ in range(2))
             ws = torch.empty(self.B.earn_beam_topk_workspace_bytes(w.batch, w.beams, vocab), dtype=torch.uint8, device=self.dev)
-            res["beam_topk"] = timed(lambda: self.B.earn_beam_topk(w.batch, w.beams, w.beams, vocab, lp, sc[0], par, tok, sc[1], ws), 1)
-            del lp, ws
+            res["beam_topk"] = timed(lambda: [self.B.earn_beam_topk(w.batch, w.beams, w.beams, vocab, lp, sc[0], par, tok, sc[1], ws)
+                                              for lp in lps], n_in)
+            del lps, ws
         if w.decode_steps > 0:
             s = w.decode_steps
             if late:

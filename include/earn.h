@@ -269,8 +269,8 @@ earn_status_t earn_train_attn_bwd(const earn_model_t* model, const earn_batch_t*
  * (zeros); parent, token: device int32 [B*W]; new_scores: device fp32 [B*W], must not alias beam_scores.
  * workspace: device, at least earn_beam_topk_workspace_bytes(batch, beams, vocab) bytes, 16-byte aligned; no need to
  * initialise it.  Errors: beams outside [1, 32], n_live outside [1, beams], n_live * vocab < beams -> INVALID_ARG;
- * beams * vocab beyond 2^31 - 1 or beyond what the two selection levels hold (3.3 M candidates at 20 beams)
- * -> UNSUPPORTED; workspace NULL / too small -> WORKSPACE. */
+ * beams * vocab beyond 2^31 - 257 (flat candidate indices are 32-bit) -> UNSUPPORTED; workspace NULL / too small
+ * -> WORKSPACE. */
 size_t earn_beam_topk_workspace_bytes(int32_t batch, int32_t beams, int32_t vocab);
 earn_status_t earn_beam_topk(int32_t batch, int32_t beams, int32_t n_live, int32_t vocab, const float* logprobs,
                              const float* beam_scores_or_null, int32_t* parent, int32_t* token, float* new_scores,

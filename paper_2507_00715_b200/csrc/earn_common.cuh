@@ -61,7 +61,7 @@ earn_status_t validate_decode(const earn_model_t* model, const earn_batch_t* bat
 void note_launch(int n = 1);
 // SMs of the current device (queried once per device); kDefaultSms when no device can be asked (host-only sizing calls)
 constexpr int kDefaultSms = 148;
-int sm_count();   // host-side count of kernels launched by this library
+int sm_count();
 
 // Opt a kernel in to `bytes` of dynamic shared memory and the largest carveout, once per device (the attribute
 // calls are not free).

@@ -152,7 +152,7 @@ def test_host_validation_beam_topk(lib):
     assert call(new=0x2000) == B.EARN_ERR_INVALID_ARG                       # the new scores would overwrite the old in place
     assert call(ws=0) == B.EARN_ERR_WORKSPACE
     assert call(beams=20, n_live=20, vocab=152064, ws_bytes=256) == B.EARN_ERR_WORKSPACE
-    assert call(beams=32, n_live=32, vocab=1 << 20) == B.EARN_ERR_UNSUPPORTED   # more chunks than the second level holds
+    assert call(beams=32, n_live=32, vocab=1 << 26) == B.EARN_ERR_UNSUPPORTED   # flat candidate indices are 32-bit
     assert call(batch=0) == B.EARN_OK
     assert lib.earn_launch_count() == n0
     # one chunk needs no partial lists; 20 beams x 152064 tokens = 372 chunks of 8192 candidates, 20 (score, index) pairs each

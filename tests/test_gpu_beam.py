@@ -80,6 +80,27 @@ def test_topk_flat_and_tied_distributions():
     check(two_valued, None, 8)
 
 
+def test_topk_values_that_keep_rising_or_arrive_late():
+    """What the running threshold of a CTA that walks several chunks must survive: scores that rise with the flat index
+    (every candidate of every later chunk beats the W-th best so far), a rise that stops half way (the pre-filter then
+    passes nothing), the best W hidden in the last chunk, equal values on both sides of a chunk boundary, and a batch
+    large enough for every CTA to take many chunks."""
+    rows, vocab, beams = 2 * 20, 40000, 20
+    rising = torch.arange(rows * vocab, device="cuda", dtype=torch.float32).reshape(rows, vocab) * 1e-3
+    check(rising - 100.0, None, beams)
+    check(-rising, None, beams)                                   # falling: only the first chunk matters
+    half = torch.minimum(rising, torch.full_like(rising, 300.0))  # rises, then a long flat top: ties by smallest index
+    check(half, None, beams)
+    w = _w(2, beams)
+    lp = wl.beam_logprobs(w, 1, vocab, "cuda")
+    lp[19, vocab - 25:] = lp.max() + 1.0 + torch.arange(25, device="cuda", dtype=torch.float32)   # the best, at the very end
+    lp[39, 8192 * 3 - 2:8192 * 3 + 2] = lp.max() + 0.5            # four equal values across a chunk boundary
+    check(lp, wl.beam_logprobs(w, 2, 7, "cuda")[:, 0].contiguous(), beams)
+    big = _w(64, beams)
+    check(wl.beam_logprobs(big, 4, 32000, "cuda"), None, beams)   # 64 x 79 chunks: a dozen chunks per CTA
+    check(wl.beam_logprobs(big, 5, 32000, "cuda"), None, beams, n_live=1)   # first decode step: one live beam, four chunks
+
+
 def test_selection_then_reparenting_then_decode():
     """A decode step whose parents come from the selection kernel: topk -> earn_beam_reparent -> earn_decode_attn on the
     device, against the oracle's selection feeding the oracle's decode state."""
