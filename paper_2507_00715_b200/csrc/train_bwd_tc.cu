@@ -20,9 +20,9 @@
 // from shared memory, or from tensor memory; right operand K-major or MN-major from a TMA-loaded tile).
 //   warp 0  TMA producer    warp 1  tcgen05.mma issuer (and TMEM owner)    warps 4-11  two softmax warpgroups, 64 columns each
 // All 512 TMEM columns are taken (X, Y, acc0, acc1), so there is no second X / Y to work ahead on; the overlap comes from
-// the issue order X(u) | acc1(u-1) | Y(u) | acc0(u): the warpgroup turns X into p while the tensor core does acc1 and Y,
-// and Y into ds while it does acc0 (issued tile by tile as X Y, then acc0 acc1, the tensor core and the warpgroup took
-// turns: 3.5 ms against the figures in the design doc for the 7B-class layer).
+// the issue order Y(u) | acc0(u) | X(u+1) | acc1(u): the warpgroups turn X(u) into p while the tensor core does acc1(u-1)
+// and Y(u), and Y(u) into ds while it does acc0(u) and X(u+1); X(u+1) only waits for p(u) to have been handed over
+// (issued tile by tile as X Y, then acc0 acc1, the tensor core and the warpgroups took turns).
 // Every mbarrier wait is bounded as in the forward kernel.
 #include "earn_common.cuh"
 #include "sm100_ptx.cuh"
@@ -218,10 +218,10 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           umma_ts_lohi(d_tmem, a_tmem + kk * 8, b_lo + kk * (2048 >> 4), desc_hi, idesc_acc, (!first || kk > 0) ? 1u : 0u);
       }
     };
-    // Order on the tensor core, per streamed tile u:  X(u) | acc1(u-1) | Y(u) | acc0(u)  -- the softmax warpgroup turns
-    // X(u) into p while acc1(u-1) and Y(u) run, and Y(u) into ds while acc0(u) runs.  One thread's tensor-core instructions
-    // run in the order they were issued, which is what lets X(u) go over the columns acc0(u-1) read p from, and Y(u)
-    // over the columns acc1(u-1) reads ds from.
+    // Order on the tensor core, per streamed tile u:  Y(u) | acc0(u) | X(u+1) | acc1(u)  -- the softmax warpgroups turn
+    // X(u) into p while acc1(u-1) and Y(u) run, and Y(u) into ds while acc0(u) and X(u+1) run.  One thread's tensor-core
+    // instructions run in the order they were issued, which is what lets X(u+1) go over the columns acc0(u) reads p
+    // from, and Y(u+1) over the columns acc1(u) reads ds from.
     bool ok = wait(C::BAR_RES, 0) && wait(C::BAR_FULL + 0, 0);
     if (ok) {
       tc_fence_after();
@@ -234,20 +234,19 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       const int st = u % C::NSTAGE, sn = (u + 1) % C::NSTAGE;
       const uint32_t t0 = sT + st * 2 * TILE, t1 = t0 + TILE, n0 = sT + sn * 2 * TILE, n1 = n0 + TILE;
       const bool more = u + 1 < job.n_iter;
-      if (MODE == MODE_KV) {
-        ok = wait(C::BAR_P, u);
-        if (!ok) break;
-        tc_fence_after();
-        issue_acc(tmem + 256, tmem + 0, t1, u == 0);      // dV += P^T dO
-      }
-      ok = wait(C::BAR_DS, u);
+      // P(u) released: MODE_KV p is in tensor memory; MODE_Q every softmax thread has its part of X(u) in registers
+      ok = wait(C::BAR_P, u);
       if (ok && more) ok = wait(C::BAR_FULL + sn, (u + 1) / C::NSTAGE);
       if (!ok) break;
       tc_fence_after();
-      if (more) {
+      if (MODE == MODE_KV) issue_acc(tmem + 256, tmem + 0, t1, u == 0);      // dV += P^T dO
+      if (more) {   // X(u+1) runs while the warpgroups are still on ds(u)
         issue_xy(tmem + 0, l_lo, smem_desc_lo(n0, 16));
         if (leader) umma_commit(bar(C::BAR_X));
       }
+      ok = wait(C::BAR_DS, u);
+      if (!ok) break;
+      tc_fence_after();
       issue_acc(tmem + 384, tmem + 128, t0, u == 0);      // dK += dS^T Q   or   dQ += dS K
       if (leader) {
         umma_commit(bar(C::BAR_EMPTY + st));
@@ -326,7 +325,12 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       tmem_ld_32x32(t_x + 32, b);
       tmem_wait_ld(a);
       tmem_wait_ld(b);
-      if (MODE == MODE_KV) asm volatile("bar.sync 2, 256;" ::: "memory");
+      if (MODE == MODE_KV) {
+        asm volatile("bar.sync 2, 256;" ::: "memory");
+      } else {   // X(u) has been read (p stays in registers): the next X may go over it
+        tc_fence_before();
+        mbar_arrive(bar(C::BAR_P));
+      }
 #pragma unroll
       for (int q = 0; q < 2; ++q) {
         uint32_t(&cur)[32] = q ? b : a;
