@@ -336,6 +336,10 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
       // Two copies of the loop, chosen once per tile: with the test for `masked` inside it, every group of four
       // columns became a basic block of its own and the pass ran at the latency of one group after another (1900
       // clocks for an interior tile, 6000 for a masked one, against 1300 for the loop without the test).
+      // the columns this lane pairs with are vis_lo .. vis_lo + vis_n - 1
+      const int vis_lo = (MODE == MODE_KV && diag) ? l : 0;
+      const int vis_hi = MODE == MODE_KV ? col_valid : (diag ? l + 1 : BM);
+      const uint32_t vis_n = (uint32_t)max(vis_hi - vis_lo, 0);
       auto p_pass = [&](auto masked_tag) {
         constexpr bool MASKED = decltype(masked_tag)::value;
 #pragma unroll
@@ -353,10 +357,8 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             e[3] = ex2(fmaf(__uint_as_float(cur[c + 3]), sl2, -ls.w));
             if (MASKED) {
 #pragma unroll
-              for (int z = 0; z < 4; ++z) {
-                const bool seen = MODE == MODE_KV ? (col + z < col_valid && (!diag || col + z >= l)) : (!diag || col + z <= l);
-                e[z] = seen ? e[z] : 0.f;
-              }
+              for (int z = 0; z < 4; ++z)   // one unsigned compare: vis_lo <= column < vis_lo + vis_n
+                e[z] = (uint32_t)(col + z - vis_lo) < vis_n ? e[z] : 0.f;
             }
             pk[q][c >> 1] = pack_bf16(e[0], e[1]);
             pk[q][(c >> 1) + 1] = pack_bf16(e[2], e[3]);
