@@ -28,6 +28,8 @@
 //
 // Every mbarrier wait is bounded; when one runs out the CTA raises its abort flag, writes
 // EARN_ERR_TIMEOUT to the status word, drains what it has in flight, frees its TMEM and returns.
+#include <type_traits>
+
 #include "earn_common.cuh"
 #include "sm100_ptx.cuh"
 #include "tc_maps.cuh"
@@ -393,32 +395,40 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             m_ref = fmaxf(mx, m1) * sl2;
           }
           const float neg_m = -m_ref;
+          // Two copies of the loop over the four chunks: an interior tile (all 128 columns visible, the usual case) takes
+          // the one without a test per chunk, which the compiler schedules as one block of straight-line code -- the end
+          // of one chunk's arithmetic overlaps the start of the next -- where the tests cut it into four.
+          auto chunks = [&](auto interior_tag) {
+            constexpr bool INTERIOR = decltype(interior_tag)::value;
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            if (q < n_chunks) {
-              uint32_t(&cur)[32] = (q & 1) ? b : a;
-              uint32_t(&nxt)[32] = (q & 1) ? a : b;
-              if (q + 1 < n_chunks) tmem_ld_32x32(t_s + (q + 1) * 32, nxt);
-              if (diag && q == wq) {
+            for (int q = 0; q < 4; ++q) {
+              if (INTERIOR || q < n_chunks) {
+                uint32_t(&cur)[32] = (q & 1) ? b : a;
+                uint32_t(&nxt)[32] = (q & 1) ? a : b;
+                if (q + 1 < 4 && (INTERIOR || q + 1 < n_chunks)) tmem_ld_32x32(t_s + (q + 1) * 32, nxt);
+                if (!INTERIOR && diag && q == wq) {
 #pragma unroll
-                for (int c = 0; c < 32; ++c)
-                  if (c > lane) cur[c] = 0xff800000u;
+                  for (int c = 0; c < 32; ++c)
+                    if (c > lane) cur[c] = 0xff800000u;
+                }
+#pragma unroll
+                for (int c = 0; c < 32; c += 2) {
+                  float e0, e1;
+                  fma2(e0, e1, __uint_as_float(cur[c]), __uint_as_float(cur[c + 1]), sl2, neg_m);
+                  e0 = ex2(e0);   // all on the special-function unit: a cubic on the FMA pipe for a share of them costs
+                  e1 = ex2(e1);   // more issue slots than it frees on the unit
+                  add2(ls0, ls1, e0, e1);
+                  pk[q][c >> 1] = pack_bf16(e0, e1);
+                }
+                if (q + 1 < 4 && (INTERIOR || q + 1 < n_chunks)) tmem_wait_ld(nxt);
+              } else {
+#pragma unroll
+                for (int c = 0; c < 16; ++c) pk[q][c] = 0u;
               }
-#pragma unroll
-              for (int c = 0; c < 32; c += 2) {
-                float e0, e1;
-                fma2(e0, e1, __uint_as_float(cur[c]), __uint_as_float(cur[c + 1]), sl2, neg_m);
-                e0 = ex2(e0);   // all on the special-function unit: moving a share of them to a cubic on the FMA pipe
-                e1 = ex2(e1);   // made the kernel slower on B200 (731 us -> 758 us per 7B layer at 6 of 16 pairs)
-                add2(ls0, ls1, e0, e1);
-                pk[q][c >> 1] = pack_bf16(e0, e1);
-              }
-              if (q + 1 < n_chunks) tmem_wait_ld(nxt);
-            } else {
-#pragma unroll
-              for (int c = 0; c < 16; ++c) pk[q][c] = 0u;
             }
-          }
+          };
+          if (n_chunks == 4 && !diag) chunks(std::true_type{});
+          else chunks(std::false_type{});
           const bool grow = !(ls0 + ls1 <= 256.f);   // also catches a sum that overflowed
           if (attempt > 0 || !__any_sync(0xffffffffu, grow)) break;
           // S_x(j) was issued after P_x V of tile j-1, so the commit that signalled it covers that too: O_x is quiescent
