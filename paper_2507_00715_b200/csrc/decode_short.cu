@@ -15,6 +15,8 @@
 //   * Eq. 4's append is served from the tile already in shared memory (no second fetch of k_new / v_new).
 // Two block-wide barriers per launch.  Everything else (which rows a lane holds, P rounded to bf16 before P V, fp32
 // accumulation, log2-domain exponentials) is as in the streaming kernels.
+#include <type_traits>
+
 #include "decode_tile.cuh"
 #include "sm100_ptx.cuh"
 
@@ -240,63 +242,79 @@ __global__ void __launch_bounds__(NW * 32) decode_short_kernel(DecodeArgs a) {
   }
   __syncthreads();
 
-  // ---- softmax of the lane's two rows over the whole list (every warp the same), P as bf16 A-fragments
-  const int n_tiles = (n_total + KT - 1) / KT;   // <= NW
-  float x0[NW][4], m0 = -INFINITY, m1 = -INFINITY;   // [tile][(r0, c2..) (r1, c2..) (r0, 8 + c2..) (r1, 8 + c2..)] pairs
-  float y0[NW][4];
+  // ---- softmax and P V, compiled once per number of key tiles in the list: with the tile count a run-time test inside
+  // the unrolled loops, every tile became a basic block of its own and its shared-memory load, exponentials and MMAs
+  // ran at their full latency one tile after another.
+  const int n_tiles = (n_total + KT - 1) / KT;   // 1 .. NW
+  float l0, l1, o[NPW][4];
+  auto tail = [&](auto n_tiles_tag) {
+    constexpr int N_TILES = decltype(n_tiles_tag)::value;
+    // ---- softmax of the lane's two rows over the whole list (every warp the same), P as bf16 A-fragments
+    float x0[NW][4], m0 = -INFINITY, m1 = -INFINITY;   // [tile][(r0, c2..) (r1, c2..) (r0, 8 + c2..) (r1, 8 + c2..)] pairs
+    float y0[NW][4];
 #pragma unroll
-  for (int kk = 0; kk < NW; ++kk) {
-    if (kk < n_tiles) {
-      const float2 a0 = *reinterpret_cast<const float2*>(sc + r0 * S::SC_PITCH + kk * KT + c2);
-      const float2 a1 = *reinterpret_cast<const float2*>(sc + r1 * S::SC_PITCH + kk * KT + c2);
-      const float2 a2 = *reinterpret_cast<const float2*>(sc + r0 * S::SC_PITCH + kk * KT + 8 + c2);
-      const float2 a3 = *reinterpret_cast<const float2*>(sc + r1 * S::SC_PITCH + kk * KT + 8 + c2);
-      x0[kk][0] = a0.x; x0[kk][1] = a0.y; x0[kk][2] = a2.x; x0[kk][3] = a2.y;
-      y0[kk][0] = a1.x; y0[kk][1] = a1.y; y0[kk][2] = a3.x; y0[kk][3] = a3.y;
-      m0 = fmaxf(m0, fmaxf(fmaxf(a0.x, a0.y), fmaxf(a2.x, a2.y)));
-      m1 = fmaxf(m1, fmaxf(fmaxf(a1.x, a1.y), fmaxf(a3.x, a3.y)));
-    }
-  }
-  m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1));
-  m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
-  m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1));
-  m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
-  if (m0 == -INFINITY) m0 = 0.f;   // a row past W*g of a list without shared rows: never stored
-  if (m1 == -INFINITY) m1 = 0.f;
-  uint32_t pf[NW][4];
-  float l0 = 0.f, l1 = 0.f;
-#pragma unroll
-  for (int kk = 0; kk < NW; ++kk) {
-    if (kk < n_tiles) {
-      const float p0 = ex2(x0[kk][0] - m0), p1 = ex2(x0[kk][1] - m0), p2 = ex2(x0[kk][2] - m0), p3 = ex2(x0[kk][3] - m0);
-      const float q0 = ex2(y0[kk][0] - m1), q1 = ex2(y0[kk][1] - m1), q2 = ex2(y0[kk][2] - m1), q3 = ex2(y0[kk][3] - m1);
-      l0 += (p0 + p1) + (p2 + p3);
-      l1 += (q0 + q1) + (q2 + q3);
-      pf[kk][0] = pack2(p0, p1); pf[kk][1] = pack2(q0, q1); pf[kk][2] = pack2(p2, p3); pf[kk][3] = pack2(q2, q3);
-    }
-  }
-  l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
-  l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
-  l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
-  l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-
-  // ---- O = P V for this warp's columns [warp * D / NW, (warp + 1) * D / NW)
-  float o[NPW][4];
-#pragma unroll
-  for (int n = 0; n < NPW; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
-  const uint32_t v_lane = kv + G::TILE_B + (uint32_t)(((mat & 1) << 3) + (lane & 7)) * G::PITCH + (uint32_t)(mat >> 1) * 16 +
-                          (uint32_t)warp * (NPW * 16);
-#pragma unroll
-  for (int kk = 0; kk < NW; ++kk) {
-    if (kk < n_tiles) {
-#pragma unroll
-      for (int nn = 0; nn < NPW / 2; ++nn) {
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4_t(v_lane + kk * G::STAGE_B + nn * 32, b0, b1, b2, b3);
-        mma_bf16(o[2 * nn], pf[kk], b0, b1);
-        mma_bf16(o[2 * nn + 1], pf[kk], b2, b3);
+    for (int kk = 0; kk < NW; ++kk) {
+      if (kk < N_TILES) {
+        const float2 a0 = *reinterpret_cast<const float2*>(sc + r0 * S::SC_PITCH + kk * KT + c2);
+        const float2 a1 = *reinterpret_cast<const float2*>(sc + r1 * S::SC_PITCH + kk * KT + c2);
+        const float2 a2 = *reinterpret_cast<const float2*>(sc + r0 * S::SC_PITCH + kk * KT + 8 + c2);
+        const float2 a3 = *reinterpret_cast<const float2*>(sc + r1 * S::SC_PITCH + kk * KT + 8 + c2);
+        x0[kk][0] = a0.x; x0[kk][1] = a0.y; x0[kk][2] = a2.x; x0[kk][3] = a2.y;
+        y0[kk][0] = a1.x; y0[kk][1] = a1.y; y0[kk][2] = a3.x; y0[kk][3] = a3.y;
+        m0 = fmaxf(m0, fmaxf(fmaxf(a0.x, a0.y), fmaxf(a2.x, a2.y)));
+        m1 = fmaxf(m1, fmaxf(fmaxf(a1.x, a1.y), fmaxf(a3.x, a3.y)));
       }
     }
+    m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1));
+    m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
+    m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1));
+    m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
+    if (m0 == -INFINITY) m0 = 0.f;   // a row past W*g of a list without shared rows: never stored
+    if (m1 == -INFINITY) m1 = 0.f;
+    uint32_t pf[NW][4];
+    l0 = 0.f, l1 = 0.f;
+#pragma unroll
+    for (int kk = 0; kk < NW; ++kk) {
+      if (kk < N_TILES) {
+        const float p0 = ex2(x0[kk][0] - m0), p1 = ex2(x0[kk][1] - m0), p2 = ex2(x0[kk][2] - m0), p3 = ex2(x0[kk][3] - m0);
+        const float q0 = ex2(y0[kk][0] - m1), q1 = ex2(y0[kk][1] - m1), q2 = ex2(y0[kk][2] - m1), q3 = ex2(y0[kk][3] - m1);
+        l0 += (p0 + p1) + (p2 + p3);
+        l1 += (q0 + q1) + (q2 + q3);
+        pf[kk][0] = pack2(p0, p1); pf[kk][1] = pack2(q0, q1); pf[kk][2] = pack2(p2, p3); pf[kk][3] = pack2(q2, q3);
+      }
+    }
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+
+    // ---- O = P V for this warp's columns [warp * D / NW, (warp + 1) * D / NW)
+#pragma unroll
+    for (int n = 0; n < NPW; ++n) o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f;
+    const uint32_t v_lane = kv + G::TILE_B + (uint32_t)(((mat & 1) << 3) + (lane & 7)) * G::PITCH + (uint32_t)(mat >> 1) * 16 +
+                            (uint32_t)warp * (NPW * 16);
+#pragma unroll
+    for (int kk = 0; kk < NW; ++kk) {
+      if (kk < N_TILES) {
+#pragma unroll
+        for (int nn = 0; nn < NPW / 2; ++nn) {
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4_t(v_lane + kk * G::STAGE_B + nn * 32, b0, b1, b2, b3);
+          mma_bf16(o[2 * nn], pf[kk], b0, b1);
+          mma_bf16(o[2 * nn + 1], pf[kk], b2, b3);
+        }
+      }
+    }
+  };
+  if (n_tiles <= 1) tail(std::integral_constant<int, 1>{});
+  else if (n_tiles == 2) tail(std::integral_constant<int, 2>{});
+  else if (n_tiles == 3) tail(std::integral_constant<int, 3>{});
+  else if (NW == 4 || n_tiles == 4) tail(std::integral_constant<int, 4>{});
+  else if constexpr (NW > 4) {
+    if (n_tiles == 5) tail(std::integral_constant<int, 5>{});
+    else if (n_tiles == 6) tail(std::integral_constant<int, 6>{});
+    else if (n_tiles == 7) tail(std::integral_constant<int, 7>{});
+    else tail(std::integral_constant<int, 8>{});
   }
   if (!a.trigger_early) pdl_launch_dependents();
   const float i0 = 1.f / l0, i1 = 1.f / l1;
