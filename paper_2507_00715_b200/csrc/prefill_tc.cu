@@ -163,7 +163,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const int first = blockIdx.x, stride = gridDim.x;   // this CTA's items: first, first + stride, ...
+  // This CTA's items: the plan is dealt to the CTAs in passes of gridDim.x items, forwards and backwards in turn (the
+  // plan is sorted longest first, so dealing every pass in the same direction gives the low-numbered CTAs the longer
+  // item of every pass: 3 % more work than the mean on the long-history shapes, 15 % on the 1.5B ones).
+  const int n_cta = gridDim.x;
+  auto item_at = [&](int k) { return k * n_cta + ((k & 1) ? n_cta - 1 - (int)blockIdx.x : (int)blockIdx.x); };
   pdl_launch_dependents();
   pdl_wait();   // the plan (written by the kernel launched just before this one) and every tensor are read below
 
@@ -172,7 +176,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     if (lane == 0) {
       int e = 0;   // ring entries issued so far, over all items
       bool ok = true;
-      for (int i = first; i < p.n_items && ok; i += stride) {
+      for (int k = 0, i = item_at(0); i < p.n_items && ok; i = item_at(++k)) {
         const Item it = load_item<PAIR_TILES>(p, i);
         const int kvh = it.kvh;
         for (int t = 0; t < 2 * it.n_tiles; ++t, ++e) {
@@ -200,7 +204,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     if (lane == 0) {
       int n = 0;   // items loaded so far
       bool ok = true;
-      for (int i = first; i < p.n_items && ok; i += stride, ++n) {
+      for (int i = item_at(0); i < p.n_items && ok; i = item_at(++n)) {
         const Item it = load_item<PAIR_TILES>(p, i);
         for (int x = 0; x < NT; ++x) {
           if (n > 0 && !mbar_wait_bounded(bar(C::BAR_QFREE + x), (n - 1) & 1, abort_flag, WAIT_LIMIT)) {
@@ -260,10 +264,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       int n_item = 0;   // items started so far
       int n_p[NT];      // P_x phases consumed so far
       for (int x = 0; x < NT; ++x) n_p[x] = 0;
-      bool ok = first < p.n_items;
+      bool ok = item_at(0) < p.n_items;
       Item cur{};
       if (ok) {
-        cur = load_item<PAIR_TILES>(p, first);
+        cur = load_item<PAIR_TILES>(p, item_at(0));
         for (int x = 0; x < NT && ok; ++x) {
           ok = wait(C::BAR_QFULL + x, 0) && (x > 0 || wait_full(0));
           if (!ok) break;
@@ -271,10 +275,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
           issue_s(x, 0, cur.n_tiles == 1);
         }
       }
-      for (int i = first; i < p.n_items && ok; i += stride, ++n_item) {
-        const bool has_next = i + stride < p.n_items;
+      for (int i = item_at(0); i < p.n_items && ok; i = item_at(++n_item)) {
+        const bool has_next = item_at(n_item + 1) < p.n_items;
         Item nxt{};
-        if (has_next) nxt = load_item<PAIR_TILES>(p, i + stride);
+        if (has_next) nxt = load_item<PAIR_TILES>(p, item_at(n_item + 1));
         const int n = cur.n_tiles;
         for (int j = 0; j < n && ok; ++j) {
           for (int x = 0; x < NT && ok; ++x) {
@@ -321,7 +325,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const float sl2 = p.scale_log2;
     int n_s = 0, n_item = 0;
     bool ok = true;
-    for (int i = first; i < p.n_items && ok; i += stride, ++n_item) {
+    for (int i = item_at(0); i < p.n_items && ok; i = item_at(++n_item)) {
       const Item it = load_item<PAIR_TILES>(p, i);
       // this M-tile's share of the item, in registers (x is not a compile-time index)
       const int h = x ? it.head[1] : it.head[0], my_diag = x ? it.diag[1] : it.diag[0];
