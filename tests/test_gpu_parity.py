@@ -119,6 +119,23 @@ def test_beam_search_row_tiles_share_the_cache_pass():
                                           beams=7, decode_steps=3, r_head=4, r_tail=4))
 
 
+def test_two_row_tiles_over_a_short_list():
+    """Beams x group size between 17 and 32 over a compact cache of a few dozen positions (the paper's own multi-head
+    setting: 20 beams, one register per side, four-token identifiers).  20 and 32 beams of a multi-head model (6 and 8
+    key tiles at the last step), 18 rows left ragged by a group of 3 (the second tile mostly empty), and lists of at
+    most four tiles behind a shuffled page table."""
+    lens = tuple(20 + (i * 11) % 60 for i in range(6))
+    run_workload_and_compare(BASE.replace(seed=41, n_q_heads=8, n_kv_heads=8, lens=lens, batch=6, beams=20,
+                                          decode_steps=4, r_head=1, r_tail=1, n_layers=2, split_k=1), check_lse=False)
+    run_workload_and_compare(BASE.replace(seed=42, n_q_heads=4, n_kv_heads=4, lens=lens[:3], batch=3, beams=32,
+                                          decode_steps=3, r_head=2, r_tail=2, n_layers=2, split_k=1), check_lse=False)
+    run_workload_and_compare(BASE.replace(seed=43, n_q_heads=6, n_kv_heads=2, lens=lens[:3], batch=3, beams=6,
+                                          decode_steps=5, r_head=3, r_tail=2, n_layers=2, split_k=1), check_lse=False)
+    run_workload_and_compare(BASE.replace(seed=44, n_q_heads=4, n_kv_heads=2, lens=lens[:2], batch=2, beams=9,
+                                          decode_steps=2, r_head=4, r_tail=4, n_layers=2, split_k=1), paged_shuffle_seed=5,
+                             check_lse=False)
+
+
 def test_two_row_tiles_on_a_grid_of_many_ctas_head_dim_64():
     """20 beams of a multi-head model (two row tiles per kv head) over more (sequence, kv head) pairs than four CTAs
     per SM hold: the launch takes the shallower ring with six CTAs per SM; head_dim 64; six decode steps, so the
