@@ -118,7 +118,8 @@ int prefill_rows_per_entry(int n_q_heads, int n_kv_heads);   // query rows one p
 int prefill_plan_entries(const earn_batch_t& b, int rows);   // (sequence, block of `rows` query rows) pairs of the batch
 // One plan entry per (sequence, block of `rows` rows): {first global row, rows of the sequence from there, block index,
 // sequence}, blocks with the highest index (the longest key range) first; at most 2048 blocks per sequence.
-cudaError_t launch_tile_plan(const int32_t* cu_seqlens, int batch, int max_seqlen, int rows, void* plan, cudaStream_t st);
+cudaError_t launch_tile_plan(const int32_t* cu_seqlens, int batch, int max_seqlen, int rows, int group_seqs, void* plan,
+                             cudaStream_t st);
 // plan: device scratch of 16 bytes per plan entry, filled by a planning kernel launched ahead of the main one
 cudaError_t launch_prefill_tc(const PrefillArgs& a, int total_tokens, int plan_entries, void* plan, int32_t* status_word,
                               cudaStream_t st);
