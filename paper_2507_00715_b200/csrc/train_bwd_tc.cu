@@ -113,7 +113,9 @@ __device__ __forceinline__ Job make_job(const BwdParams& p) {
 template <int MODE>
 __global__ void __launch_bounds__(BCfg::THREADS, 1)
 train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                    const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do, BwdParams p) {
+                    const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
+                    const __grid_constant__ CUtensorMap map_out0, const __grid_constant__ CUtensorMap map_out1, BwdParams p) {
+  // map_out0 / map_out1: MODE_KV dV and dK, MODE_Q unused and dQ (boxes of 32 rows x 64 columns, one per warp)
   using C = BCfg;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -143,6 +145,8 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     tma_prefetch_desc(&map_k);
     tma_prefetch_desc(&map_v);
     tma_prefetch_desc(&map_do);
+    tma_prefetch_desc(&map_out0);
+    tma_prefetch_desc(&map_out1);
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), C::TMEM_COLS);
@@ -431,6 +435,43 @@ train_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           }
         }
       };
+      // A whole tile of the sequence leaves through shared memory and the copy engine instead (each thread writing its
+      // own row with 16-byte stores puts 2048 half-sector writes per accumulator through the SM's one load/store unit:
+      // about 3600 clocks, a quarter of a dQ item).  The resident pair's 64 KB are free once the last product has
+      // retired: warp (wg, wq) stages its 32 rows x 64 columns there, 128-byte swizzled, and its first lane hands the
+      // slab to the copy engine.  `slot` tells the two accumulators of MODE_KV apart.
+      auto store_tile = [&](uint32_t t_acc, const CUtensorMap* map, int head, float mul, int slot) {
+        const uint32_t out = sL + (uint32_t)(slot * 8 + (warp - 4)) * (32 * 128);
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          tmem_ld_32x32(t_acc + c0 + q * 32, a);
+          tmem_wait_ld(a);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {   // 16-byte chunk q * 4 + c of the lane's 128-byte row, at chunk ^ (row % 8)
+            const uint32_t w0 = pack_bf16(__uint_as_float(a[c * 8 + 0]) * mul, __uint_as_float(a[c * 8 + 1]) * mul);
+            const uint32_t w1 = pack_bf16(__uint_as_float(a[c * 8 + 2]) * mul, __uint_as_float(a[c * 8 + 3]) * mul);
+            const uint32_t w2 = pack_bf16(__uint_as_float(a[c * 8 + 4]) * mul, __uint_as_float(a[c * 8 + 5]) * mul);
+            const uint32_t w3 = pack_bf16(__uint_as_float(a[c * 8 + 6]) * mul, __uint_as_float(a[c * 8 + 7]) * mul);
+            const int ch = q * 4 + c;
+            st_shared_v4(out + (uint32_t)lane * 128 + (uint32_t)((ch ^ (lane & 7)) << 4), w0, w1, w2, w3);
+          }
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_3d(map, out, c0, head, job.left_row0 + wq * 32);
+          bulk_commit();
+        }
+      };
+      if (job.left_valid == BM) {
+        if (MODE == MODE_KV) {
+          store_tile(t_lane + 256, &map_out0, job.kvh, 1.f, 0);
+          store_tile(t_lane + 384, &map_out1, job.kvh, p.scale, 1);
+        } else {
+          store_tile(t_lane + 384, &map_out1, job.head0, p.scale, 0);
+        }
+        if (lane == 0) bulk_wait_all0();   // the copies have completed before the CTA gives its shared memory back
+      } else
       if (MODE == MODE_KV) {
         store_rows(t_lane + 256, p.dv, p.Hkv, job.kvh, 1.f);
         store_rows(t_lane + 384, p.dk, p.Hkv, job.kvh, p.scale);
@@ -509,9 +550,11 @@ bool train_bwd_tc_supported(const TrainArgs& a) {
 
 cudaError_t launch_train_bwd_tc(const TrainArgs& a, const earn_batch_t& b, void* plan, cudaStream_t st) {
   using tcmap::make_map;
-  CUtensorMap mq, mk, mv, mdo;
+  CUtensorMap mq, mk, mv, mdo, mdq, mdk, mdv;
   if (!make_map(&mq, a.q, a.Hq, a.total, BM) || !make_map(&mk, a.k, a.Hkv, a.total, BM) ||
-      !make_map(&mv, a.v, a.Hkv, a.total, BM) || !make_map(&mdo, a.d_o, a.Hq, a.total, BM))
+      !make_map(&mv, a.v, a.Hkv, a.total, BM) || !make_map(&mdo, a.d_o, a.Hq, a.total, BM) ||
+      !make_map(&mdq, a.dq, a.Hq, a.total, 32) || !make_map(&mdk, a.dk, a.Hkv, a.total, 32) ||
+      !make_map(&mdv, a.dv, a.Hkv, a.total, 32))   // gradients leave in slabs of 32 rows, one per warp
     return cudaErrorInvalidValue;
   const int n_entries = prefill_plan_entries(b, BM);
   if (n_entries <= 0) return cudaSuccess;
@@ -534,14 +577,14 @@ cudaError_t launch_train_bwd_tc(const TrainArgs& a, const earn_batch_t& b, void*
   e = ensure_dynamic_smem<train_bwd_tc_kernel<MODE_KV>>(BCfg::SMEM_BYTES);
   if (e == cudaSuccess)
     e = launch_pdl(train_bwd_tc_kernel<MODE_KV>, dim3((unsigned)((int64_t)n_entries * a.Hkv)), dim3(BCfg::THREADS),
-                   BCfg::SMEM_BYTES, st, mq, mk, mv, mdo, p);
+                   BCfg::SMEM_BYTES, st, mq, mk, mv, mdo, mdv, mdk, p);
   note_launch();
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   e = ensure_dynamic_smem<train_bwd_tc_kernel<MODE_Q>>(BCfg::SMEM_BYTES);
   if (e == cudaSuccess)
     e = launch_pdl(train_bwd_tc_kernel<MODE_Q>, dim3((unsigned)((int64_t)n_entries * a.Hq)), dim3(BCfg::THREADS),
-                   BCfg::SMEM_BYTES, st, mq, mk, mv, mdo, p);
+                   BCfg::SMEM_BYTES, st, mq, mk, mv, mdo, mdq, mdq, p);
   note_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }
