@@ -356,14 +356,17 @@ cudaError_t launch_decode_mma(const DecodeArgs& a0, int max_shared_len, cudaStre
   const long ctas = (long)(a.plan.n_splits > 0 ? a.plan.n_splits : 1) * a.plan.row_tiles * a.Hkv * a.batch;
   const bool unsplit = a.plan.n_splits <= 1;
   const bool four_warps = unsplit && max_tiles <= 16 && ctas < sm_count();
+  // a longer list on such a grid (the planner leaves it unsplit up to kDecodeUnsplitMaxLen shared positions): eight warps
+  const bool eight_warps = unsplit && !four_warps && ctas < sm_count() && max_shared_len <= kDecodeUnsplitMaxLen;
   // a list of one or two tiles goes into a three-stage ring whole; anything longer is walked in pairs
   const bool two_tiles = unsplit && max_tiles <= 2;
   if (a.D == 64)
-    return four_warps  ? launch_d<64, 2, 4, SHARED>(a, st)
+    return four_warps  ? launch_d<64, 2, 4, SHARED>(a, st)   // (the planner only leaves such a list unsplit at head_dim 128)
            : two_tiles ? launch_d<64, 3, 1, SHORT>(a, st)
                         : launch_d<64, EARN_DECODE_STAGES, 1, STREAM>(a, st);
-  return four_warps  ? launch_d<128, 2, 4, SHARED>(a, st)
-         : two_tiles ? launch_d<128, 3, 1, SHORT>(a, st)
+  return four_warps    ? launch_d<128, 2, 4, SHARED>(a, st)
+         : eight_warps ? launch_d<128, 2, 8, SHARED>(a, st)
+         : two_tiles   ? launch_d<128, 3, 1, SHORT>(a, st)
                       : launch_d<128, EARN_DECODE_STAGES, 1, STREAM>(a, st);
 }
 

@@ -45,6 +45,7 @@ struct DecodePlan {
   int n_splits;    // ceil(max shared length / chunk); 0 when the shared segment is empty
 };
 constexpr int kDecodeRows = 16;
+constexpr int kDecodeUnsplitMaxLen = 2048;   // shared positions a grid of less than one CTA per SM walks without split-KV
 DecodePlan make_decode_plan(const earn_model_t& m, const earn_batch_t& b, int beams, int max_shared_len);
 size_t decode_partial_floats(const earn_model_t& m, const earn_batch_t& b, const DecodePlan& p);
 
