@@ -116,10 +116,13 @@ __global__ void __launch_bounds__(NW * 32) decode_short_kernel(DecodeArgs a) {
   int64_t p_off[PASSES];
   int p_key[PASSES];
 #pragma unroll
+  for (int i = 0; i < PASSES; ++i) {   // (all table reads first, in one block of code: they overlap)
+    p_off[i] = tab_off[r_t + i * RPP] + c_t * 8;
+    p_key[i] = tab_key[r_t + i * RPP];
+  }
+#pragma unroll
   for (int i = 0; i < PASSES; ++i) {
     const int p = r_t + i * RPP;
-    p_off[i] = tab_off[p] + c_t * 8;
-    p_key[i] = tab_key[p];
     if (p < n_shared) {
       cp_async16(dst_of(p), kg + p_off[i]);
       cp_async16(dst_of(p) + G::TILE_B, vg + p_off[i]);
