@@ -9,6 +9,8 @@
 // asynchronous copies (in flight together with the K/V copies), reads them back as ldmatrix
 // fragments, runs mma.sync m16n8k16 over 16-key tiles up to the causal limit with an online softmax
 // in the log2 domain, and writes its 16 output rows through the same private tile as 16-byte stores.
+#include <type_traits>
+
 #include "earn_common.cuh"
 #include "mma_sync.cuh"
 #include "sm100_ptx.cuh"
@@ -141,6 +143,67 @@ __global__ void __launch_bounds__(NW * 32, 12 / NW) register_mma_kernel(Register
 #pragma unroll
     for (int n = 0; n < NTILES; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
 
+    // At most 32 registers (one or two key tiles, the usual case): all scores first, one maximum, one round of
+    // exponentials, then P V with nothing to rescale -- compiled for the tile count, so that the whole tile is one block
+    // of straight-line code.  Longer register lists take the running-maximum loop below.
+    auto short_list = [&](auto tiles_tag) {
+      constexpr int KTS = decltype(tiles_tag)::value;
+      float s[KTS][2][4];
+#pragma unroll
+      for (int kt = 0; kt < KTS; ++kt) {
+#pragma unroll
+        for (int n = 0; n < 2; ++n) s[kt][n][0] = s[kt][n][1] = s[kt][n][2] = s[kt][n][3] = 0.f;
+        const uint32_t ks = sK + kt * 16 * G::PITCH;
+#pragma unroll
+        for (int kk = 0; kk < KSTEPS; ++kk) {
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4(ks + k_lane + kk * 32, b0, b1, b2, b3);
+          mma_bf16(s[kt][0], qf[kk], b0, b1);
+          mma_bf16(s[kt][1], qf[kk], b2, b3);
+        }
+      }
+      float t0 = -INFINITY, t1 = -INFINITY;
+#pragma unroll
+      for (int kt = 0; kt < KTS; ++kt)
+#pragma unroll
+        for (int n = 0; n < 2; ++n)
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int j = kt * 16 + n * 8 + c2 + (e & 1);
+            s[kt][n][e] = j > ((e < 2) ? m0r : m1r) ? -INFINITY : s[kt][n][e];   // key after the row's own register (also j >= R)
+            if (e < 2) t0 = fmaxf(t0, s[kt][n][e]); else t1 = fmaxf(t1, s[kt][n][e]);
+          }
+      t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, 1));
+      t0 = fmaxf(t0, __shfl_xor_sync(0xffffffffu, t0, 2));
+      t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, 1));
+      t1 = fmaxf(t1, __shfl_xor_sync(0xffffffffu, t1, 2));
+      const float mu0 = t0 * scale_log2, mu1 = t1 * scale_log2;   // every row sees at least key 0: finite
+      uint32_t pf[KTS][4];
+#pragma unroll
+      for (int kt = 0; kt < KTS; ++kt) {
+        const float p00 = ex2(fmaf(s[kt][0][0], scale_log2, -mu0)), p01 = ex2(fmaf(s[kt][0][1], scale_log2, -mu0));
+        const float p02 = ex2(fmaf(s[kt][0][2], scale_log2, -mu1)), p03 = ex2(fmaf(s[kt][0][3], scale_log2, -mu1));
+        const float p10 = ex2(fmaf(s[kt][1][0], scale_log2, -mu0)), p11 = ex2(fmaf(s[kt][1][1], scale_log2, -mu0));
+        const float p12 = ex2(fmaf(s[kt][1][2], scale_log2, -mu1)), p13 = ex2(fmaf(s[kt][1][3], scale_log2, -mu1));
+        l0 += p00 + p01 + p10 + p11;
+        l1 += p02 + p03 + p12 + p13;
+        pf[kt][0] = pack2(p00, p01); pf[kt][1] = pack2(p02, p03); pf[kt][2] = pack2(p10, p11); pf[kt][3] = pack2(p12, p13);
+      }
+#pragma unroll
+      for (int kt = 0; kt < KTS; ++kt) {
+        const uint32_t vs = sV + kt * 16 * G::PITCH;
+#pragma unroll
+        for (int nn = 0; nn < NTILES / 2; ++nn) {
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4_t(vs + v_lane + nn * 32, b0, b1, b2, b3);
+          mma_bf16(o[2 * nn], pf[kt], b0, b1);
+          mma_bf16(o[2 * nn + 1], pf[kt], b2, b3);
+        }
+      }
+    };
+    if (key_tiles == 1) short_list(std::integral_constant<int, 1>{});
+    else if (key_tiles == 2) short_list(std::integral_constant<int, 2>{});
+    else
     for (int kt = 0; kt < key_tiles; ++kt) {
       const uint32_t ks = sK + kt * 16 * G::PITCH, vs = sV + kt * 16 * G::PITCH;
       float s[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
