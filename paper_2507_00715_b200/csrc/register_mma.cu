@@ -31,8 +31,13 @@ struct RGeo {
   static constexpr int PITCH = ROWB + 16;
 };
 
-template <int D, int NW>
-__global__ void __launch_bounds__(NW * 32, 12 / NW) register_mma_kernel(RegisterArgs a, int r_pad) {
+// Four CTAs of four warps per SM (MINB = 4: 128 registers, 16 bytes of spills): the 512 CTAs of the 7B shapes are then
+// resident at once instead of 1.15 waves of three per SM (18.4 -> 14.7 us per fused register layer; 28.8 -> 27.4
+// ragged).  The eight-warp form, which runs on small grids, keeps all the registers it wants when every CTA has an SM to
+// itself (capped, it lost 0.7 us at the 1.5B shapes) and is held to two CTAs per SM when there are more CTAs than SMs
+// (192 CTAs: 6.1 -> 4.4 us, one wave instead of two).
+template <int D, int NW, int MINB>
+__global__ void __launch_bounds__(NW * 32, MINB) register_mma_kernel(RegisterArgs a, int r_pad) {
   using bf16 = __nv_bfloat16;
   using G = RGeo<D>;
   constexpr int KSTEPS = D / 16, NTILES = D / 8, CH = G::ROWB / 16;
@@ -282,14 +287,14 @@ __global__ void __launch_bounds__(NW * 32, 12 / NW) register_mma_kernel(Register
   }
 }
 
-template <int D, int NW>
+template <int D, int NW, int MINB>
 cudaError_t launch_r(const RegisterArgs& a, cudaStream_t st) {
   const int r_pad = (a.R + 15) / 16 * 16;
   const int smem = 2 * r_pad * RGeo<D>::PITCH + NW * 16 * RGeo<D>::PITCH;
-  cudaError_t e = ensure_dynamic_smem<register_mma_kernel<D, NW>>(2 * MAX_R * RGeo<D>::PITCH + NW * 16 * RGeo<D>::PITCH);
+  cudaError_t e = ensure_dynamic_smem<register_mma_kernel<D, NW, MINB>>(2 * MAX_R * RGeo<D>::PITCH + NW * 16 * RGeo<D>::PITCH);
   if (e != cudaSuccess) return e;
   dim3 grid(a.Hkv, a.batch);
-  e = launch_pdl(register_mma_kernel<D, NW>, grid, dim3(NW * 32), smem, st, a, r_pad);
+  e = launch_pdl(register_mma_kernel<D, NW, MINB>, grid, dim3(NW * 32), smem, st, a, r_pad);
   note_launch();
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -299,9 +304,11 @@ cudaError_t launch_r(const RegisterArgs& a, cudaStream_t st) {
 bool register_mma_supported(const RegisterArgs& a) { return a.dtype == EARN_BF16 && a.R <= MAX_R; }
 
 cudaError_t launch_register_mma(const RegisterArgs& a, cudaStream_t st) {
-  const bool small_grid = (long)a.Hkv * a.batch <= 2L * sm_count();
-  if (a.D == 64) return small_grid ? launch_r<64, 8>(a, st) : launch_r<64, 4>(a, st);
-  return small_grid ? launch_r<128, 8>(a, st) : launch_r<128, 4>(a, st);
+  const long ctas = (long)a.Hkv * a.batch;
+  const bool small_grid = ctas <= 2L * sm_count(), one_each = ctas <= sm_count();
+  if (a.D == 64)
+    return !small_grid ? launch_r<64, 4, 4>(a, st) : one_each ? launch_r<64, 8, 1>(a, st) : launch_r<64, 8, 2>(a, st);
+  return !small_grid ? launch_r<128, 4, 4>(a, st) : one_each ? launch_r<128, 8, 1>(a, st) : launch_r<128, 8, 2>(a, st);
 }
 
 }  // namespace earn
